@@ -1,0 +1,270 @@
+// Persistent, warp-specialised tcgen05 GEMM engine for sm_100a.
+//
+//   D[M, N] = A[M, K] * B[N, K]^T      bf16 operands, fp32 accumulation in TMEM
+//
+// One CTA per SM, 192 threads:
+//   warp 0      TMA producer (one lane): global -> 128B-swizzled shared tiles
+//   warp 1      MMA issuer (one lane): tcgen05.mma, accumulators in TMEM
+//   warps 2..5  epilogue: tcgen05.ld the 128 x BN fp32 tile and hand it to `Epi`
+// The accumulator is double-buffered in TMEM (2 x BN columns) so the epilogue of
+// tile j overlaps the MMAs of tile j+1.  The shared-memory ring has STAGES slots
+// of (128 x 64) A + (BN x 64) B.
+//
+// Either operand may be "K-major" (contraction index contiguous in global
+// memory: the tensor map's inner dimension is K) or "MN-major" (the M or N index
+// contiguous: the tensor map's inner dimension is M/N and its outer one is K).
+//
+// Work is cut into units: a unit is one 128-row tile and a contiguous range of
+// BN-wide column tiles.  The epilogue keeps per-thread state across the tiles of
+// a unit (e.g. a running max / sum-exp), which is how the vocabulary reduction
+// is fused without ever storing the logits.
+#pragma once
+#include <cuda.h>
+#include <cuda_runtime.h>
+#include <cstdint>
+
+#include "ptx.cuh"
+
+namespace cpmtp {
+
+constexpr int kBM = 128;          // rows per tile = TMEM lanes
+constexpr int kBK = 64;           // bf16 elements per 128-byte swizzle row
+constexpr int kGemmThreads = 192;
+constexpr int kEpiThreads = 128;
+
+// Values raised in the device status word.
+constexpr int kDevOk = 0;
+constexpr int kDevTargetOutOfRange = 1;
+constexpr int kDevWaitTimeout = 2;
+
+struct Sched {
+  int m_tiles;    // number of 128-row tiles
+  int n_tiles;    // number of BN-column tiles
+  int n_splits;   // column tiles are cut into this many contiguous ranges
+  int m_group;    // row tiles that are swept together (L2 locality)
+  int k_blocks;   // contraction length / 64, rounded up
+  int units;      // ceil(m_tiles / m_group) * m_group * n_splits
+};
+
+inline Sched make_sched(int m_tiles, int n_tiles, int n_splits, int m_group, int k_blocks) {
+  Sched s;
+  if (n_splits > n_tiles) n_splits = n_tiles;
+  if (n_splits < 1) n_splits = 1;
+  if (m_group > m_tiles) m_group = m_tiles;
+  if (m_group < 1) m_group = 1;
+  s.m_tiles = m_tiles;
+  s.n_tiles = n_tiles;
+  s.n_splits = n_splits;
+  s.m_group = m_group;
+  s.k_blocks = k_blocks;
+  s.units = ((m_tiles + m_group - 1) / m_group) * m_group * n_splits;
+  return s;
+}
+
+// Unit u -> (row tile, split, column-tile range).  Consecutive units (which run
+// concurrently on neighbouring CTAs) walk the row tiles of one group first.
+__device__ __forceinline__ bool decode_unit(const Sched& s, int u, int& m_tile, int& split,
+                                            int& n_begin, int& n_end) {
+  const int per_group = s.m_group * s.n_splits;
+  const int g = u / per_group;
+  const int rem = u - g * per_group;
+  split = rem / s.m_group;
+  m_tile = g * s.m_group + (rem - split * s.m_group);
+  if (m_tile >= s.m_tiles) return false;
+  n_begin = static_cast<int>((static_cast<long long>(split) * s.n_tiles) / s.n_splits);
+  n_end = static_cast<int>((static_cast<long long>(split + 1) * s.n_tiles) / s.n_splits);
+  return n_end > n_begin;
+}
+
+template <int BN_, int STAGES_, bool A_MN_, bool B_MN_>
+struct TileCfg {
+  static constexpr int BN = BN_;
+  static constexpr int STAGES = STAGES_;
+  static constexpr bool A_MN = A_MN_;
+  static constexpr bool B_MN = B_MN_;
+  static constexpr int A_BYTES = kBM * kBK * 2;
+  static constexpr int B_BYTES = BN * kBK * 2;
+  static constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
+  static constexpr int TMEM_COLS = (2 * BN <= 32) ? 32 : (2 * BN <= 64) ? 64 : (2 * BN <= 128) ? 128
+                                   : (2 * BN <= 256) ? 256 : 512;
+  static_assert(BN % 16 == 0 && BN >= 16 && BN <= 256, "MMA N must be a multiple of 16 in [16, 256]");
+  static_assert(!B_MN || BN % 64 == 0, "an MN-major B tile is loaded in 64-wide boxes");
+  static_assert(STAGE_BYTES % 1024 == 0, "stages must keep 1024-byte alignment for the swizzle");
+};
+
+constexpr int kBarrierBytes = 256;
+
+template <class Cfg, class Epi>
+constexpr int gemm_smem_bytes() {
+  return 1024 + Cfg::STAGES * Cfg::STAGE_BYTES + kBarrierBytes + Epi::SMEM_BYTES;
+}
+
+template <class Cfg, class Epi>
+__global__ void __launch_bounds__(kGemmThreads, 1)
+tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
+               const Sched sched, const typename Epi::Params ep, int* __restrict__ dev_status) {
+  extern __shared__ uint8_t smem_raw[];
+  const uint32_t raw_addr = ptx::smem_u32(smem_raw);
+  const uint32_t pad = (1024u - (raw_addr & 1023u)) & 1023u;
+  uint8_t* smem = smem_raw + pad;
+  const uint32_t tiles_addr = raw_addr + pad;
+  uint8_t* bar_mem = smem + Cfg::STAGES * Cfg::STAGE_BYTES;
+  const uint32_t bar_addr = tiles_addr + Cfg::STAGES * Cfg::STAGE_BYTES;
+  // barrier layout (8 bytes each): full[STAGES], empty[STAGES], tfull[2], tempty[2], drain
+  auto full_bar = [&](int s) { return bar_addr + 8u * s; };
+  auto empty_bar = [&](int s) { return bar_addr + 8u * (Cfg::STAGES + s); };
+  auto tfull_bar = [&](int a) { return bar_addr + 8u * (2 * Cfg::STAGES + a); };
+  auto tempty_bar = [&](int a) { return bar_addr + 8u * (2 * Cfg::STAGES + 2 + a); };
+  const uint32_t drain_bar = bar_addr + 8u * (2 * Cfg::STAGES + 4);
+  static_assert(8 * (2 * Cfg::STAGES + 5) + 16 <= kBarrierBytes, "barrier area too small");
+  volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(bar_mem + kBarrierBytes - 16);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(bar_mem + kBarrierBytes - 8);
+  uint8_t* epi_smem = bar_mem + kBarrierBytes;
+
+  const int warp = threadIdx.x >> 5;
+  const int lane = threadIdx.x & 31;
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < Cfg::STAGES; ++s) {
+      ptx::mbar_init(full_bar(s), 1);
+      ptx::mbar_init(empty_bar(s), 1);
+    }
+    for (int a = 0; a < 2; ++a) {
+      ptx::mbar_init(tfull_bar(a), 1);
+      ptx::mbar_init(tempty_bar(a), kEpiThreads);
+    }
+    ptx::mbar_init(drain_bar, 1);
+    *abort_flag = 0;
+    ptx::fence_mbar_init();
+    ptx::prefetch_tmap(&tmA);
+    ptx::prefetch_tmap(&tmB);
+  }
+  if (warp == 1) {
+    ptx::tmem_alloc(ptx::smem_u32(const_cast<uint32_t*>(tmem_slot)), Cfg::TMEM_COLS);
+    ptx::tmem_relinquish();
+  }
+  ptx::tc_fence_before_sync();
+  __syncthreads();
+  ptx::tc_fence_after_sync();
+  const uint32_t tmem_base = *tmem_slot;
+
+  if (warp == 0) {
+    // ------------------------------------------------------------ producer
+    if (lane == 0) {
+      int it = 0;
+      bool alive = true;
+      for (int u = blockIdx.x; u < sched.units && alive; u += gridDim.x) {
+        int m_tile, split, n_begin, n_end;
+        if (!decode_unit(sched, u, m_tile, split, n_begin, n_end)) continue;
+        for (int nt = n_begin; nt < n_end && alive; ++nt) {
+          for (int kb = 0; kb < sched.k_blocks; ++kb, ++it) {
+            const int s = it % Cfg::STAGES;
+            const uint32_t ph = (it / Cfg::STAGES) & 1;
+            if (!ptx::mbar_wait(empty_bar(s), ph ^ 1u, abort_flag)) { alive = false; break; }
+            ptx::mbar_arrive_expect_tx(full_bar(s), Cfg::STAGE_BYTES);
+            const uint32_t a_dst = tiles_addr + s * Cfg::STAGE_BYTES;
+            const uint32_t b_dst = a_dst + Cfg::A_BYTES;
+            if constexpr (!Cfg::A_MN) {
+              ptx::tma_load_2d(a_dst, &tmA, full_bar(s), kb * kBK, m_tile * kBM);
+            } else {
+#pragma unroll
+              for (int j = 0; j < kBM / 64; ++j)
+                ptx::tma_load_2d(a_dst + j * 8192, &tmA, full_bar(s), m_tile * kBM + j * 64, kb * kBK);
+            }
+            if constexpr (!Cfg::B_MN) {
+              ptx::tma_load_2d(b_dst, &tmB, full_bar(s), kb * kBK, nt * Cfg::BN);
+            } else {
+#pragma unroll
+              for (int j = 0; j < Cfg::BN / 64; ++j)
+                ptx::tma_load_2d(b_dst + j * 8192, &tmB, full_bar(s), nt * Cfg::BN + j * 64, kb * kBK);
+            }
+          }
+        }
+      }
+      // Drain: every load issued must have landed before this CTA's shared memory is released.
+      const int issued = it;
+      for (int back = 1; back <= Cfg::STAGES && back <= issued; ++back) {
+        const int j = issued - back;
+        ptx::mbar_wait(full_bar(j % Cfg::STAGES), (j / Cfg::STAGES) & 1, abort_flag, false);
+      }
+    }
+  } else if (warp == 1) {
+    // ---------------------------------------------------------- MMA issuer
+    if (lane == 0) {
+      constexpr uint32_t idesc = ptx::make_idesc_bf16(kBM, Cfg::BN, Cfg::A_MN ? 1 : 0, Cfg::B_MN ? 1 : 0);
+      constexpr uint32_t a_kstep = Cfg::A_MN ? 2048u : 32u;   // bytes per 16-element K step
+      constexpr uint32_t b_kstep = Cfg::B_MN ? 2048u : 32u;
+      // K-major: 8-row groups are 1024 B apart (stride offset); the leading offset is unused.
+      // MN-major: 64-element blocks along M/N are 8192 B apart (leading offset), 8-row K groups 1024 B.
+      constexpr uint32_t a_lbo = Cfg::A_MN ? 8192u : 16u;
+      constexpr uint32_t b_lbo = Cfg::B_MN ? 8192u : 16u;
+      int it = 0, acc_it = 0;
+      bool alive = true;
+      for (int u = blockIdx.x; u < sched.units && alive; u += gridDim.x) {
+        int m_tile, split, n_begin, n_end;
+        if (!decode_unit(sched, u, m_tile, split, n_begin, n_end)) continue;
+        for (int nt = n_begin; nt < n_end && alive; ++nt, ++acc_it) {
+          const int acc = acc_it & 1;
+          const uint32_t acc_ph = (acc_it >> 1) & 1;
+          if (!ptx::mbar_wait(tempty_bar(acc), acc_ph ^ 1u, abort_flag)) { alive = false; break; }
+          ptx::tc_fence_after_sync();
+          const uint32_t d_tmem = tmem_base + acc * Cfg::BN;
+          for (int kb = 0; kb < sched.k_blocks; ++kb, ++it) {
+            const int s = it % Cfg::STAGES;
+            const uint32_t ph = (it / Cfg::STAGES) & 1;
+            if (!ptx::mbar_wait(full_bar(s), ph, abort_flag)) { alive = false; break; }
+            ptx::tc_fence_after_sync();
+            const uint32_t a_src = tiles_addr + s * Cfg::STAGE_BYTES;
+            const uint32_t b_src = a_src + Cfg::A_BYTES;
+#pragma unroll
+            for (int kk = 0; kk < kBK / 16; ++kk) {
+              const uint64_t adesc = ptx::make_smem_desc_sw128(a_src + kk * a_kstep, a_lbo, 1024);
+              const uint64_t bdesc = ptx::make_smem_desc_sw128(b_src + kk * b_kstep, b_lbo, 1024);
+              ptx::umma_bf16(d_tmem, adesc, bdesc, idesc, (kb | kk) != 0 ? 1u : 0u);
+            }
+            ptx::umma_commit(empty_bar(s));   // frees the slot once these MMAs have read it
+          }
+          if (alive) ptx::umma_commit(tfull_bar(acc));
+        }
+      }
+      // Drain: all issued MMAs must retire before TMEM is freed.
+      ptx::umma_commit(drain_bar);
+      ptx::mbar_wait(drain_bar, 0, abort_flag, false);
+    }
+  } else {
+    // ------------------------------------------------------------ epilogue
+    // These waits ignore the other roles' abort flag: all four warps wait on the
+    // same barrier, so they either all pass or all time out, and no warp is left
+    // alone at a barrier an epilogue might use internally.
+    const int quarter = warp & 3;                 // TMEM lane quarter this warp may read
+    const int row_in_tile = quarter * 32 + lane;
+    const int epi_tid = threadIdx.x - 64;
+    typename Epi::State st;
+    int acc_it = 0;
+    bool alive = true;
+    for (int u = blockIdx.x; u < sched.units && alive; u += gridDim.x) {
+      int m_tile, split, n_begin, n_end;
+      if (!decode_unit(sched, u, m_tile, split, n_begin, n_end)) continue;
+      Epi::unit_begin(ep, st, m_tile, split, row_in_tile);
+      for (int nt = n_begin; nt < n_end; ++nt, ++acc_it) {
+        const int acc = acc_it & 1;
+        const uint32_t acc_ph = (acc_it >> 1) & 1;
+        if (!ptx::mbar_wait(tfull_bar(acc), acc_ph, abort_flag, false)) { alive = false; break; }
+        ptx::tc_fence_after_sync();
+        const uint32_t tacc = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16) + acc * Cfg::BN;
+        Epi::tile(ep, st, tacc, m_tile, nt, row_in_tile, epi_smem, epi_tid);
+        ptx::tc_fence_before_sync();
+        ptx::mbar_arrive(tempty_bar(acc));
+      }
+      if (alive) Epi::unit_end(ep, st, m_tile, split, row_in_tile, epi_smem, epi_tid);
+    }
+  }
+
+  ptx::tc_fence_before_sync();
+  __syncthreads();
+  ptx::tc_fence_after_sync();
+  if (warp == 1) ptx::tmem_dealloc(tmem_base, Cfg::TMEM_COLS);
+  if (threadIdx.x == 0 && *abort_flag != 0 && dev_status != nullptr) atomicMax(dev_status, kDevWaitTimeout);
+}
+
+}  // namespace cpmtp
