@@ -1,0 +1,154 @@
+/*
+ * cpmtp — fused log-likelihood of a rank-r canonical-polyadic (CP) multi-token
+ * prediction head, for NVIDIA B200 (sm_100a).
+ *
+ * The joint distribution of the next n tokens is modelled as a mixture of r
+ * experts, each a product of n per-token softmax factors (Eq. 2, Eq. 3), with
+ * mixture weights from a gate (Eq. 7) and factors from per-(token, expert)
+ * head projections followed by a shared unembedding (Eq. 6 in its reduced,
+ * shared-head form from the fine-tuning section):
+ *
+ *   w[i, :]        = softmax(W_g h[i])                                   (Eq. 7)
+ *   S[i, s, a, :]  = E (W_head[s*r + a] h[i])                            (Eq. 6, shared head)
+ *   C[i, s, a]     = S[i, s, a, x[i, s]] - logsumexp_v S[i, s, a, v]     (Eq. 8)
+ *   logp[i]        = logsumexp_a( log w[i, a] + sum_s C[i, s, a] )       (Eq. 9)
+ *
+ * Conventions for every entry point
+ *  - All tensor pointers are DEVICE pointers owned by the caller unless a
+ *    parameter is documented as a host pointer.  Row-major, densely packed.
+ *    bf16 tensors are passed as `const void*` / `void*` (2 bytes per element)
+ *    and must be 16-byte aligned; fp32 / int32 tensors 4-byte aligned.
+ *  - The library allocates and frees no device memory; scratch space is the
+ *    caller's `workspace`, sized by cpmtp_workspace_bytes(), 256-byte aligned.
+ *    Work is enqueued on `stream` and is asynchronous with respect to the host.
+ *  - Return value: CPMTP_OK or a negative error code; on a validation error
+ *    nothing was enqueued.  `dev_status` (device int32, may be NULL; the caller
+ *    zeroes it) is raised by kernels to 1 if a target token was outside [0, V)
+ *    (the token is clamped, the run continues) or 2 if an internal bounded wait
+ *    expired (results invalid).
+ *  - Limits: d % 64 == 0, 1 <= r <= 32, 1 <= n <= 8, N >= 1, V >= 2,
+ *    N*n*r*d < 2^40.
+ */
+#ifndef CPMTP_H
+#define CPMTP_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define CPMTP_MAX_R 32
+#define CPMTP_MAX_N 8
+
+enum {
+  CPMTP_OK = 0,
+  CPMTP_ERR_NULL = -1,      /* a required pointer is NULL */
+  CPMTP_ERR_SHAPE = -2,     /* sizes outside the limits above */
+  CPMTP_ERR_ALIGN = -3,     /* a pointer is not aligned as required */
+  CPMTP_ERR_WORKSPACE = -4, /* workspace_bytes too small */
+  CPMTP_ERR_ARCH = -5,      /* current device is not compute capability 10.x */
+  CPMTP_ERR_LAUNCH = -6,    /* a CUDA call failed; see cudaGetLastError */
+  CPMTP_ERR_LIMIT = -7      /* size beyond a fixed built-in capacity */
+};
+
+enum { CPMTP_OP_FORWARD = 0, CPMTP_OP_BACKWARD = 1, CPMTP_OP_SCORE = 2 };
+
+/* flags */
+#define CPMTP_FLAG_AUX 1u /* add aux_coef * sum_a wbar_a^2 to the loss (soft form of Eq. 10) */
+
+typedef struct cpmtp_shape {
+  int32_t N;        /* positions */
+  int32_t d;        /* embedding size (the paper's E) */
+  int32_t V;        /* vocabulary size */
+  int32_t n;        /* tokens predicted per position */
+  int32_t r;        /* CP rank = number of experts */
+  uint32_t flags;   /* CPMTP_FLAG_* */
+  float aux_coef;   /* weight of the balance term, used when CPMTP_FLAG_AUX is set */
+} cpmtp_shape;
+
+/* Forward results kept for the backward pass; every pointer is a caller-owned
+ * device buffer of the stated size. */
+typedef struct cpmtp_saved {
+  float* lse;   /* [N, n*r]  logsumexp_v S                       */
+  float* tgt;   /* [N, n*r]  S at the target token               */
+  float* logw;  /* [N, r]    log gate weights (Eq. 7)            */
+  float* q;     /* [N, r]    expert posterior exp(a - logp)      */
+  float* wbar;  /* [r]       mean gate weight over positions     */
+  void* z;      /* [N, n*r, d] bf16 projected hidden states      */
+} cpmtp_saved;
+
+typedef struct CUstream_st* cpmtp_stream;
+
+int cpmtp_version(void);
+const char* cpmtp_status_string(int status);
+
+/* Scratch bytes needed by `op` (CPMTP_OP_*) for this shape; 0 if the shape is invalid. */
+size_t cpmtp_workspace_bytes(const cpmtp_shape* shape, int op);
+
+/*
+ * Joint log-likelihood per position, logp[i] of Eq. 9, with the vocabulary
+ * reduction of Eq. 8 fused into the unembedding so that the logits are never
+ * written to memory.
+ *   h [N,d] bf16, W_head [n*r,d,d] bf16 (k = s*r + a, [out][in]), E [V,d] bf16,
+ *   W_g [r,d] bf16, x [N,n] int32 targets.
+ *   logp [N] fp32 out.
+ *   loss [1] fp32 out or NULL: -(1/N) sum_i logp[i] (+ aux_coef * sum_a wbar_a^2 with CPMTP_FLAG_AUX).
+ *   saved: NULL for inference, else filled for cpmtp_backward.
+ *   expert_counts [r] int32 out or NULL: n_a of Eq. 10, the number of positions
+ *     whose largest gate weight is expert a (ties to the lowest a).
+ */
+int cpmtp_forward(const cpmtp_shape* shape, const void* h, const void* W_head, const void* E,
+                  const void* W_g, const int32_t* x, float* logp, float* loss,
+                  const cpmtp_saved* saved, int32_t* expert_counts, void* workspace,
+                  size_t workspace_bytes, int32_t* dev_status, cpmtp_stream stream);
+
+/*
+ * Gradient of  sum_i u[i] * logp[i] (+ the balance term with CPMTP_FLAG_AUX)
+ * with respect to h, W_head, E and W_g (chain rule through Eq. 9, Eq. 8, Eq. 7);
+ * u = dloss_dlogp [N] fp32, or NULL for u[i] = -1/N (the mean negative
+ * log-likelihood that training minimises).  The logits are recomputed tile by
+ * tile from `saved` (as filled by cpmtp_forward on the same inputs).  Outputs are
+ * bf16, rounded once from fp32 accumulators:
+ *   dh [N,d], dW_head [n*r,d,d], dE [V,d], dW_g [r,d]; all required.
+ */
+int cpmtp_backward(const cpmtp_shape* shape, const void* h, const void* W_head, const void* E,
+                   const void* W_g, const int32_t* x, const cpmtp_saved* saved,
+                   const float* dloss_dlogp, void* dh, void* dW_head, void* dE, void* dW_g,
+                   void* workspace, size_t workspace_bytes, int32_t* dev_status,
+                   cpmtp_stream stream);
+
+/*
+ * Score a given draft for verification (speculative-decoding section): the same
+ * quantity as cpmtp_forward for a small number of positions, tuned for the
+ * memory-bound regime where E and W_head are each streamed once.
+ *   draft [N,n] int32.  logp_joint [N] fp32 out.
+ *   logp_prefix [N,n] fp32 out or NULL: log P(draft[i, 0..s]) for s = 0..n-1,
+ *   the mixture with only the first s+1 factors folded into the expert weights
+ *   (sampling section; s = 0 is Eq. 11).
+ */
+int cpmtp_score_draft(const cpmtp_shape* shape, const void* h, const void* W_head, const void* E,
+                      const void* W_g, const int32_t* draft, float* logp_joint, float* logp_prefix,
+                      void* workspace, size_t workspace_bytes, int32_t* dev_status,
+                      cpmtp_stream stream);
+
+/*
+ * cpmtp_forward with the per-step operands in HOST memory: h_host [N,d] bf16 and
+ * x_host [N,n] int32 (pinned memory recommended) are copied to the device, the
+ * forward pass of Eq. 9 runs, and logp_host [N] / loss_host [1] (either may be
+ * NULL) are copied back, all on `stream`.  Weights stay device-resident.  The
+ * workspace must hold cpmtp_workspace_bytes(shape, CPMTP_OP_FORWARD) plus
+ * cpmtp_host_staging_bytes(shape) bytes.  Returns after enqueueing: synchronise
+ * the stream before reading the host outputs.
+ */
+size_t cpmtp_host_staging_bytes(const cpmtp_shape* shape);
+int cpmtp_forward_host(const cpmtp_shape* shape, const void* h_host, const void* W_head,
+                       const void* E, const void* W_g, const int32_t* x_host, float* logp_host,
+                       float* loss_host, const cpmtp_saved* saved, void* workspace,
+                       size_t workspace_bytes, int32_t* dev_status, cpmtp_stream stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* CPMTP_H */
