@@ -1,0 +1,220 @@
+"""ctypes binding of libcpmtp.so: argument marshalling only.
+
+Every step of the computation runs in the library's CUDA kernels; torch is used
+for device memory and the current stream.  There is no fallback: if the shared
+library is missing or fails to load, importing this module's functions raises.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from dataclasses import dataclass
+from typing import Optional
+
+import torch
+
+from .build import LIB_PATH
+
+OP_FORWARD, OP_BACKWARD, OP_SCORE = 0, 1, 2
+FLAG_AUX = 1
+
+EXPORTS = [
+    "cpmtp_version", "cpmtp_status_string", "cpmtp_workspace_bytes", "cpmtp_forward", "cpmtp_backward",
+    "cpmtp_score_draft", "cpmtp_host_staging_bytes", "cpmtp_forward_host",
+]
+
+
+class CShape(ctypes.Structure):
+    _fields_ = [("N", ctypes.c_int32), ("d", ctypes.c_int32), ("V", ctypes.c_int32), ("n", ctypes.c_int32),
+                ("r", ctypes.c_int32), ("flags", ctypes.c_uint32), ("aux_coef", ctypes.c_float)]
+
+
+class CSaved(ctypes.Structure):
+    _fields_ = [("lse", ctypes.c_void_p), ("tgt", ctypes.c_void_p), ("logw", ctypes.c_void_p),
+                ("q", ctypes.c_void_p), ("wbar", ctypes.c_void_p), ("z", ctypes.c_void_p)]
+
+
+_lib = None
+
+
+def load_library() -> ctypes.CDLL:
+    """Load libcpmtp.so (built in-tree by build.py); raise if it is absent."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    if not os.path.exists(LIB_PATH):
+        raise RuntimeError(f"{LIB_PATH} not found: build it with `python -m paper_2410_17765_b200.build`")
+    lib = ctypes.CDLL(LIB_PATH)
+    vp, sz, i32p, fp = ctypes.c_void_p, ctypes.c_size_t, ctypes.c_void_p, ctypes.c_void_p
+    shp = ctypes.POINTER(CShape)
+    svp = ctypes.POINTER(CSaved)
+    lib.cpmtp_version.restype = ctypes.c_int
+    lib.cpmtp_status_string.restype = ctypes.c_char_p
+    lib.cpmtp_status_string.argtypes = [ctypes.c_int]
+    lib.cpmtp_workspace_bytes.restype = sz
+    lib.cpmtp_workspace_bytes.argtypes = [shp, ctypes.c_int]
+    lib.cpmtp_host_staging_bytes.restype = sz
+    lib.cpmtp_host_staging_bytes.argtypes = [shp]
+    lib.cpmtp_forward.restype = ctypes.c_int
+    lib.cpmtp_forward.argtypes = [shp, vp, vp, vp, vp, i32p, fp, fp, svp, i32p, vp, sz, i32p, vp]
+    lib.cpmtp_backward.restype = ctypes.c_int
+    lib.cpmtp_backward.argtypes = [shp, vp, vp, vp, vp, i32p, svp, fp, vp, vp, vp, vp, vp, sz, i32p, vp]
+    lib.cpmtp_score_draft.restype = ctypes.c_int
+    lib.cpmtp_score_draft.argtypes = [shp, vp, vp, vp, vp, i32p, fp, fp, vp, sz, i32p, vp]
+    lib.cpmtp_forward_host.restype = ctypes.c_int
+    lib.cpmtp_forward_host.argtypes = [shp, vp, vp, vp, vp, i32p, fp, fp, svp, vp, sz, i32p, vp]
+    _lib = lib
+    return lib
+
+
+class CpmtpError(RuntimeError):
+    pass
+
+
+def _check(rc: int) -> None:
+    if rc != 0:
+        raise CpmtpError(f"cpmtp error {rc}: {load_library().cpmtp_status_string(rc).decode()}")
+
+
+def _ptr(t: Optional[torch.Tensor]):
+    return None if t is None else ctypes.c_void_p(t.data_ptr())
+
+
+def _stream():
+    return ctypes.c_void_p(torch.cuda.current_stream().cuda_stream)
+
+
+def make_shape(N, d, V, n, r, aux_coef: Optional[float] = None) -> CShape:
+    flags = FLAG_AUX if aux_coef is not None else 0
+    return CShape(N, d, V, n, r, flags, float(aux_coef or 0.0))
+
+
+def workspace_bytes(shape: CShape, op: int) -> int:
+    return int(load_library().cpmtp_workspace_bytes(ctypes.byref(shape), op))
+
+
+def host_staging_bytes(shape: CShape) -> int:
+    return int(load_library().cpmtp_host_staging_bytes(ctypes.byref(shape)))
+
+
+def alloc_workspace(nbytes: int, device="cuda") -> torch.Tensor:
+    return torch.empty(max(nbytes, 256), dtype=torch.uint8, device=device)
+
+
+@dataclass
+class Saved:
+    """Forward results kept for cpmtp_backward (device tensors)."""
+    lse: torch.Tensor
+    tgt: torch.Tensor
+    logw: torch.Tensor
+    q: torch.Tensor
+    wbar: torch.Tensor
+    z: torch.Tensor
+
+    @staticmethod
+    def alloc(shape: CShape, device="cuda") -> "Saved":
+        K = shape.n * shape.r
+        f = dict(dtype=torch.float32, device=device)
+        return Saved(lse=torch.empty((shape.N, K), **f), tgt=torch.empty((shape.N, K), **f),
+                     logw=torch.empty((shape.N, shape.r), **f), q=torch.empty((shape.N, shape.r), **f),
+                     wbar=torch.empty((32,), **f),
+                     z=torch.empty((shape.N, K, shape.d), dtype=torch.bfloat16, device=device))
+
+    def c_struct(self) -> CSaved:
+        return CSaved(self.lse.data_ptr(), self.tgt.data_ptr(), self.logw.data_ptr(), self.q.data_ptr(),
+                      self.wbar.data_ptr(), self.z.data_ptr())
+
+
+def _shape_of(h, W_head, E, W_g, x, aux_coef) -> CShape:
+    N, d = h.shape
+    V = E.shape[0]
+    n = x.shape[1]
+    r = W_g.shape[0]
+    assert W_head.shape == (n * r, d, d) and E.shape[1] == d and W_g.shape[1] == d and x.shape[0] == N
+    for t in (h, W_head, E, W_g):
+        assert t.dtype == torch.bfloat16 and t.is_contiguous()
+    assert x.dtype == torch.int32 and x.is_contiguous()
+    return make_shape(N, d, V, n, r, aux_coef)
+
+
+def forward(h, W_head, E, W_g, x, *, aux_coef: Optional[float] = None, saved: Optional[Saved] = None,
+            want_loss: bool = True, want_counts: bool = False, workspace: Optional[torch.Tensor] = None,
+            dev_status: Optional[torch.Tensor] = None, out: Optional[dict] = None) -> dict:
+    """cpmtp_forward on device tensors; returns {"logp", "loss", "counts"} (device tensors)."""
+    lib = load_library()
+    shape = _shape_of(h, W_head, E, W_g, x, aux_coef)
+    dev = h.device
+    if workspace is None:
+        workspace = alloc_workspace(workspace_bytes(shape, OP_FORWARD), dev)
+    res = out if out is not None else {}
+    if "logp" not in res:
+        res["logp"] = torch.empty(shape.N, dtype=torch.float32, device=dev)
+    if want_loss and "loss" not in res:
+        res["loss"] = torch.empty(1, dtype=torch.float32, device=dev)
+    if want_counts and "counts" not in res:
+        res["counts"] = torch.empty(shape.r, dtype=torch.int32, device=dev)
+    cs = saved.c_struct() if saved is not None else None
+    rc = lib.cpmtp_forward(ctypes.byref(shape), _ptr(h), _ptr(W_head), _ptr(E), _ptr(W_g), _ptr(x),
+                           _ptr(res["logp"]), _ptr(res.get("loss")) if want_loss else None,
+                           ctypes.byref(cs) if cs is not None else None,
+                           _ptr(res.get("counts")) if want_counts else None, _ptr(workspace),
+                           workspace.numel(), _ptr(dev_status), _stream())
+    _check(rc)
+    return res
+
+
+def backward(h, W_head, E, W_g, x, saved: Saved, *, aux_coef: Optional[float] = None,
+             dloss_dlogp: Optional[torch.Tensor] = None, workspace: Optional[torch.Tensor] = None,
+             dev_status: Optional[torch.Tensor] = None, out: Optional[dict] = None) -> dict:
+    """cpmtp_backward on device tensors; returns {"dh", "dW_head", "dE", "dW_g"} (bf16 device tensors)."""
+    lib = load_library()
+    shape = _shape_of(h, W_head, E, W_g, x, aux_coef)
+    if workspace is None:
+        workspace = alloc_workspace(workspace_bytes(shape, OP_BACKWARD), h.device)
+    res = out if out is not None else {}
+    for name, ref in (("dh", h), ("dW_head", W_head), ("dE", E), ("dW_g", W_g)):
+        if name not in res:
+            res[name] = torch.empty_like(ref)
+    cs = saved.c_struct()
+    rc = lib.cpmtp_backward(ctypes.byref(shape), _ptr(h), _ptr(W_head), _ptr(E), _ptr(W_g), _ptr(x),
+                            ctypes.byref(cs), _ptr(dloss_dlogp), _ptr(res["dh"]), _ptr(res["dW_head"]),
+                            _ptr(res["dE"]), _ptr(res["dW_g"]), _ptr(workspace), workspace.numel(),
+                            _ptr(dev_status), _stream())
+    _check(rc)
+    return res
+
+
+def score_draft(h, W_head, E, W_g, draft, *, want_prefix: bool = True,
+                workspace: Optional[torch.Tensor] = None, dev_status: Optional[torch.Tensor] = None,
+                out: Optional[dict] = None) -> dict:
+    """cpmtp_score_draft; returns {"logp_joint", "logp_prefix"} (device tensors)."""
+    lib = load_library()
+    shape = _shape_of(h, W_head, E, W_g, draft, None)
+    if workspace is None:
+        workspace = alloc_workspace(workspace_bytes(shape, OP_SCORE), h.device)
+    res = out if out is not None else {}
+    if "logp_joint" not in res:
+        res["logp_joint"] = torch.empty(shape.N, dtype=torch.float32, device=h.device)
+    if want_prefix and "logp_prefix" not in res:
+        res["logp_prefix"] = torch.empty((shape.N, shape.n), dtype=torch.float32, device=h.device)
+    rc = lib.cpmtp_score_draft(ctypes.byref(shape), _ptr(h), _ptr(W_head), _ptr(E), _ptr(W_g), _ptr(draft),
+                               _ptr(res["logp_joint"]), _ptr(res.get("logp_prefix")) if want_prefix else None,
+                               _ptr(workspace), workspace.numel(), _ptr(dev_status), _stream())
+    _check(rc)
+    return res
+
+
+def forward_host(h_host, W_head, E, W_g, x_host, logp_host, loss_host, *, aux_coef: Optional[float] = None,
+                 workspace: Optional[torch.Tensor] = None, dev_status: Optional[torch.Tensor] = None) -> None:
+    """cpmtp_forward_host: h_host / x_host / logp_host / loss_host are (pinned) CPU tensors; weights on device.
+    Asynchronous: synchronise the current stream before reading the host outputs."""
+    lib = load_library()
+    N, d = h_host.shape
+    shape = make_shape(N, d, E.shape[0], x_host.shape[1], W_g.shape[0], aux_coef)
+    need = workspace_bytes(shape, OP_FORWARD) + host_staging_bytes(shape) + 256
+    if workspace is None:
+        workspace = alloc_workspace(need, E.device)
+    rc = lib.cpmtp_forward_host(ctypes.byref(shape), _ptr(h_host), _ptr(W_head), _ptr(E), _ptr(W_g), _ptr(x_host),
+                                _ptr(logp_host), _ptr(loss_host), None, _ptr(workspace), workspace.numel(),
+                                _ptr(dev_status), _stream())
+    _check(rc)

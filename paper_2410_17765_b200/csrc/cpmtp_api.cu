@@ -1,0 +1,443 @@
+// C-ABI of the CP-head log-likelihood library: validation, workspace layout and
+// the launch sequence of each entry point.  See include/cpmtp.h for the contract.
+#include "../../include/cpmtp.h"
+
+#include <cuda.h>
+#include <cuda_runtime.h>
+#include <cstdint>
+#include <cstdlib>
+
+#include "epilogues.cuh"
+#include "small_kernels.cuh"
+#include "tc_gemm.cuh"
+#include "tmap.cuh"
+
+namespace cpmtp {
+namespace {
+
+constexpr int kBN = 256;
+constexpr int kStages = 4;
+constexpr size_t kAlign = 256;
+constexpr size_t kLogitGradBudgetBytes = 4ull << 30;   // bound on the recomputed-logit-gradient chunk
+
+using CfgKK = TileCfg<kBN, kStages, false, false>;   // A K-major, B K-major
+using CfgKM = TileCfg<kBN, kStages, false, true>;    // A K-major, B MN-major
+using CfgMM = TileCfg<kBN, kStages, true, true>;     // both MN-major
+
+inline size_t align_up(size_t v, size_t a = kAlign) { return (v + a - 1) / a * a; }
+
+struct DeviceInfo {
+  int sms = 0;
+  int cc_major = 0;
+  bool ok = false;
+};
+
+// Cached per device ordinal; filled on first use with that device current.
+DeviceInfo* device_info() {
+  static DeviceInfo infos[64];
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return nullptr;
+  DeviceInfo& di = infos[dev];
+  if (!di.ok) {
+    if (cudaDeviceGetAttribute(&di.sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return nullptr;
+    if (cudaDeviceGetAttribute(&di.cc_major, cudaDevAttrComputeCapabilityMajor, dev) != cudaSuccess)
+      return nullptr;
+    di.ok = true;
+  }
+  return &di;
+}
+
+int validate_shape(const cpmtp_shape* s) {
+  if (s == nullptr) return CPMTP_ERR_NULL;
+  if (s->N < 1 || s->d < 64 || s->V < 2 || s->n < 1 || s->r < 1) return CPMTP_ERR_SHAPE;
+  if (s->d % 64 != 0 || s->r > CPMTP_MAX_R || s->n > CPMTP_MAX_N) return CPMTP_ERR_SHAPE;
+  const double zsize = static_cast<double>(s->N) * s->n * s->r * s->d;
+  if (zsize >= 1099511627776.0) return CPMTP_ERR_SHAPE;
+  if (static_cast<double>(s->N) * s->n * s->r >= 2147483648.0) return CPMTP_ERR_SHAPE;
+  return CPMTP_OK;
+}
+
+inline bool aligned(const void* p, size_t a) { return (reinterpret_cast<uintptr_t>(p) % a) == 0; }
+
+// Column-split schedule of the fused unembedding: `group` row tiles x `splits`
+// vocabulary ranges run concurrently, so the rows' z tiles stay L2-resident while
+// each range of E is streamed once per group.
+Sched sched_lse(int m_tiles, int n_tiles, int k_blocks, int sms) {
+  int splits, group;
+  if (m_tiles >= sms) {
+    splits = n_tiles < 4 ? n_tiles : 4;
+    group = sms / splits;
+  } else {
+    splits = (sms + m_tiles - 1) / m_tiles;
+    if (splits > n_tiles) splits = n_tiles;
+    group = m_tiles;
+  }
+  return make_sched(m_tiles, n_tiles, splits, group, k_blocks);
+}
+
+struct FwdLayout {
+  size_t logw, q, wbar, lse, tgt, z, tgt_part, part_m, part_l, total;
+  Sched lse_sched;
+  int K, M;   // heads, rows of the unembedding GEMM
+};
+
+FwdLayout fwd_layout(const cpmtp_shape& s, int sms) {
+  FwdLayout L;
+  L.K = s.n * s.r;
+  L.M = s.N * L.K;
+  const int m_tiles = (L.M + kBM - 1) / kBM;
+  const int n_tiles = (s.V + kBN - 1) / kBN;
+  L.lse_sched = sched_lse(m_tiles, n_tiles, s.d / kBK, sms);
+  size_t off = 0;
+  auto take = [&](size_t bytes) { size_t o = off; off = align_up(off + bytes); return o; };
+  L.logw = take(sizeof(float) * s.N * s.r);
+  L.q = take(sizeof(float) * s.N * s.r);
+  L.wbar = take(sizeof(float) * CPMTP_MAX_R);
+  L.lse = take(sizeof(float) * L.M);
+  L.tgt = take(sizeof(float) * L.M);
+  L.z = take(2ull * L.M * s.d);
+  L.tgt_part = take(sizeof(float) * static_cast<size_t>(L.M) * (s.d / 64));
+  L.part_m = take(sizeof(float) * static_cast<size_t>(L.M) * L.lse_sched.n_splits);
+  L.part_l = take(sizeof(float) * static_cast<size_t>(L.M) * L.lse_sched.n_splits);
+  L.total = off;
+  return L;
+}
+
+struct BwdLayout {
+  size_t coef, dg, dz, G, dE32, dwg_part, total;
+  int K, M, ldg, chunk_rows, chunks, dwg_slices, dwg_rows_per_slice;
+};
+
+BwdLayout bwd_layout(const cpmtp_shape& s) {
+  BwdLayout L;
+  L.K = s.n * s.r;
+  L.M = s.N * L.K;
+  L.ldg = (s.V + 63) / 64 * 64;
+  long long rows = static_cast<long long>(kLogitGradBudgetBytes / (2ull * L.ldg)) / kBM * kBM;
+  if (const char* env = std::getenv("CPMTP_BWD_CHUNK_ROWS")) {
+    const long long v = std::atoll(env);
+    if (v >= kBM) rows = v / kBM * kBM;
+  }
+  if (rows < kBM) rows = kBM;
+  const long long m_pad = (static_cast<long long>(L.M) + kBM - 1) / kBM * kBM;
+  if (rows > m_pad) rows = m_pad;
+  L.chunk_rows = static_cast<int>(rows);
+  L.chunks = static_cast<int>((L.M + rows - 1) / rows);
+  L.dwg_rows_per_slice = 256;
+  L.dwg_slices = (s.N + L.dwg_rows_per_slice - 1) / L.dwg_rows_per_slice;
+  size_t off = 0;
+  auto take = [&](size_t bytes) { size_t o = off; off = align_up(off + bytes); return o; };
+  L.coef = take(sizeof(float) * s.N * s.r);
+  L.dg = take(sizeof(float) * s.N * s.r);
+  L.dz = take(2ull * L.M * s.d);
+  L.G = take(2ull * L.chunk_rows * L.ldg);
+  L.dE32 = take(L.chunks > 1 ? sizeof(float) * static_cast<size_t>(s.V) * s.d : 0);
+  L.dwg_part = take(sizeof(float) * static_cast<size_t>(L.dwg_slices) * s.r * s.d);
+  L.total = off;
+  return L;
+}
+
+template <class Cfg, class Epi>
+cudaError_t launch_gemm(const void* A, uint64_t a_rows, uint64_t a_ld, const void* B, uint64_t b_rows,
+                        uint64_t b_ld, uint64_t kdim, const Sched& sched, const typename Epi::Params& ep,
+                        int* dev_status, int sms, cudaStream_t stream) {
+  static bool attr_set[64] = {};
+  CUtensorMap tA, tB;
+  if (!make_operand_tmap(&tA, A, Cfg::A_MN, a_rows, kdim, a_ld, kBM)) return cudaErrorInvalidValue;
+  if (!make_operand_tmap(&tB, B, Cfg::B_MN, b_rows, kdim, b_ld, Cfg::BN)) return cudaErrorInvalidValue;
+  constexpr int smem = gemm_smem_bytes<Cfg, Epi>();
+  int dev = 0;
+  cudaGetDevice(&dev);
+  if (dev >= 0 && dev < 64 && !attr_set[dev]) {
+    cudaError_t e = cudaFuncSetAttribute(tc_gemm_kernel<Cfg, Epi>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+    if (e != cudaSuccess) return e;
+    attr_set[dev] = true;
+  }
+  const int grid = sched.units < sms ? sched.units : sms;
+  tc_gemm_kernel<Cfg, Epi><<<grid, kGemmThreads, smem, stream>>>(tA, tB, sched, ep, dev_status);
+  return cudaGetLastError();
+}
+
+#define CPMTP_TRY(expr)                         \
+  do {                                          \
+    if ((expr) != cudaSuccess) return CPMTP_ERR_LAUNCH; \
+  } while (0)
+
+// Forward pipeline shared by cpmtp_forward and cpmtp_score_draft.
+int run_forward(const cpmtp_shape& s, const uint16_t* h, const uint16_t* W_head, const uint16_t* E,
+                const uint16_t* W_g, const int32_t* x, float* logp, float* loss, const cpmtp_saved* saved,
+                int32_t* counts, float* logp_prefix, uint8_t* ws, const FwdLayout& L, int* dev_status, int sms,
+                cudaStream_t stream) {
+  float* logw = saved ? saved->logw : reinterpret_cast<float*>(ws + L.logw);
+  float* q = saved ? saved->q : reinterpret_cast<float*>(ws + L.q);
+  float* wbar = saved ? saved->wbar : reinterpret_cast<float*>(ws + L.wbar);
+  float* lse = saved ? saved->lse : reinterpret_cast<float*>(ws + L.lse);
+  float* tgt = saved ? saved->tgt : reinterpret_cast<float*>(ws + L.tgt);
+  uint16_t* z = saved ? static_cast<uint16_t*>(saved->z) : reinterpret_cast<uint16_t*>(ws + L.z);
+  float* tgt_part = reinterpret_cast<float*>(ws + L.tgt_part);
+  float* part_m = reinterpret_cast<float*>(ws + L.part_m);
+  float* part_l = reinterpret_cast<float*>(ws + L.part_l);
+  const int K = L.K;
+  const int ncols = K * s.d;
+
+  // gate (Eq. 7)
+  {
+    const int warps = 8;
+    gate_kernel<<<(s.N + warps - 1) / warps, warps * 32, 0, stream>>>(h, W_g, logw, s.N, s.d, s.r);
+    CPMTP_TRY(cudaGetLastError());
+  }
+  // head projection: z[N, K*d] = h[N, d] * W_cat[K*d, d]^T, plus the fp32 target-logit partials
+  {
+    EpiProj<kBN>::Params ep{z, tgt_part, E, x, dev_status, s.N, ncols, s.d, s.V, s.n, s.r};
+    const int m_tiles = (s.N + kBM - 1) / kBM;
+    const int n_tiles = (ncols + kBN - 1) / kBN;
+    const Sched sc = make_sched(m_tiles, n_tiles, n_tiles, m_tiles < 64 ? m_tiles : 64, s.d / kBK);
+    CPMTP_TRY((launch_gemm<CfgKK, EpiProj<kBN>>(h, s.N, s.d, W_head, ncols, s.d, s.d, sc, ep, dev_status, sms, stream)));
+  }
+  // unembedding fused with the vocabulary log-sum-exp (Eq. 6, Eq. 8)
+  {
+    EpiLse<kBN>::Params ep{part_m, part_l, L.M, s.V, L.lse_sched.n_splits};
+    CPMTP_TRY((launch_gemm<CfgKK, EpiLse<kBN>>(z, L.M, s.d, E, s.V, s.d, s.d, L.lse_sched, ep, dev_status, sms, stream)));
+  }
+  // mixture epilogue (Eq. 9)
+  {
+    const int warps = 8;
+    mixture_kernel<<<(s.N + warps - 1) / warps, warps * 32, 0, stream>>>(
+        part_m, part_l, L.lse_sched.n_splits, tgt_part, s.d / 64, logw, lse, tgt, q, logp, logp_prefix, s.N, s.n, s.r);
+    CPMTP_TRY(cudaGetLastError());
+  }
+  if (loss != nullptr || counts != nullptr || saved != nullptr) {
+    const float aux = (s.flags & CPMTP_FLAG_AUX) ? s.aux_coef : 0.f;
+    finalize_kernel<<<1, 1024, 0, stream>>>(logp, logw, wbar, counts, loss, s.N, s.r, aux);
+    CPMTP_TRY(cudaGetLastError());
+  }
+  return CPMTP_OK;
+}
+
+int check_common(const cpmtp_shape* shape, const void* h, const void* W_head, const void* E, const void* W_g,
+                 const void* x, const void* workspace, DeviceInfo** di_out) {
+  const int vs = validate_shape(shape);
+  if (vs != CPMTP_OK) return vs;
+  if (!h || !W_head || !E || !W_g || !x || !workspace) return CPMTP_ERR_NULL;
+  if (!aligned(h, 16) || !aligned(W_head, 16) || !aligned(E, 16) || !aligned(W_g, 16) || !aligned(x, 4) ||
+      !aligned(workspace, kAlign))
+    return CPMTP_ERR_ALIGN;
+  DeviceInfo* di = device_info();
+  if (di == nullptr) return CPMTP_ERR_LAUNCH;
+  if (di->cc_major != 10) return CPMTP_ERR_ARCH;
+  *di_out = di;
+  return CPMTP_OK;
+}
+
+int check_saved(const cpmtp_saved* sv) {
+  if (!sv->lse || !sv->tgt || !sv->logw || !sv->q || !sv->wbar || !sv->z) return CPMTP_ERR_NULL;
+  if (!aligned(sv->z, 16) || !aligned(sv->lse, 4) || !aligned(sv->tgt, 4) || !aligned(sv->logw, 4) ||
+      !aligned(sv->q, 4) || !aligned(sv->wbar, 4))
+    return CPMTP_ERR_ALIGN;
+  return CPMTP_OK;
+}
+
+}  // namespace
+}  // namespace cpmtp
+
+using namespace cpmtp;
+
+static int sms_or_default() {
+  DeviceInfo* di = device_info();
+  return (di != nullptr && di->sms > 0) ? di->sms : 148;
+}
+
+extern "C" {
+
+int cpmtp_version(void) { return 100; }
+
+const char* cpmtp_status_string(int status) {
+  switch (status) {
+    case CPMTP_OK: return "ok";
+    case CPMTP_ERR_NULL: return "a required pointer is NULL";
+    case CPMTP_ERR_SHAPE: return "shape outside the supported limits (d % 64 == 0, r <= 32, n <= 8, sizes >= 1)";
+    case CPMTP_ERR_ALIGN: return "a pointer is not aligned as required";
+    case CPMTP_ERR_WORKSPACE: return "workspace too small";
+    case CPMTP_ERR_ARCH: return "current device is not compute capability 10.x";
+    case CPMTP_ERR_LAUNCH: return "a CUDA call failed";
+    case CPMTP_ERR_LIMIT: return "size beyond a fixed built-in capacity";
+    default: return "unknown status";
+  }
+}
+
+size_t cpmtp_workspace_bytes(const cpmtp_shape* shape, int op) {
+  if (validate_shape(shape) != CPMTP_OK) return 0;
+  const int sms = sms_or_default();
+  switch (op) {
+    case CPMTP_OP_FORWARD:
+    case CPMTP_OP_SCORE: return fwd_layout(*shape, sms).total;
+    case CPMTP_OP_BACKWARD: return bwd_layout(*shape).total;
+    default: return 0;
+  }
+}
+
+size_t cpmtp_host_staging_bytes(const cpmtp_shape* shape) {
+  if (validate_shape(shape) != CPMTP_OK) return 0;
+  return align_up(2ull * shape->N * shape->d) + align_up(4ull * shape->N * shape->n) +
+         align_up(4ull * shape->N) + align_up(4);
+}
+
+int cpmtp_forward(const cpmtp_shape* shape, const void* h, const void* W_head, const void* E, const void* W_g,
+                  const int32_t* x, float* logp, float* loss, const cpmtp_saved* saved, int32_t* expert_counts,
+                  void* workspace, size_t workspace_bytes, int32_t* dev_status, cpmtp_stream stream) {
+  DeviceInfo* di = nullptr;
+  const int rc = check_common(shape, h, W_head, E, W_g, x, workspace, &di);
+  if (rc != CPMTP_OK) return rc;
+  if (logp == nullptr) return CPMTP_ERR_NULL;
+  if (saved != nullptr) {
+    const int rs = check_saved(saved);
+    if (rs != CPMTP_OK) return rs;
+  }
+  const FwdLayout L = fwd_layout(*shape, di->sms);
+  if (workspace_bytes < L.total) return CPMTP_ERR_WORKSPACE;
+  return run_forward(*shape, static_cast<const uint16_t*>(h), static_cast<const uint16_t*>(W_head),
+                     static_cast<const uint16_t*>(E), static_cast<const uint16_t*>(W_g), x, logp, loss, saved,
+                     expert_counts, nullptr, static_cast<uint8_t*>(workspace), L, dev_status, di->sms,
+                     reinterpret_cast<cudaStream_t>(stream));
+}
+
+int cpmtp_score_draft(const cpmtp_shape* shape, const void* h, const void* W_head, const void* E,
+                      const void* W_g, const int32_t* draft, float* logp_joint, float* logp_prefix,
+                      void* workspace, size_t workspace_bytes, int32_t* dev_status, cpmtp_stream stream) {
+  DeviceInfo* di = nullptr;
+  const int rc = check_common(shape, h, W_head, E, W_g, draft, workspace, &di);
+  if (rc != CPMTP_OK) return rc;
+  if (logp_joint == nullptr) return CPMTP_ERR_NULL;
+  const FwdLayout L = fwd_layout(*shape, di->sms);
+  if (workspace_bytes < L.total) return CPMTP_ERR_WORKSPACE;
+  return run_forward(*shape, static_cast<const uint16_t*>(h), static_cast<const uint16_t*>(W_head),
+                     static_cast<const uint16_t*>(E), static_cast<const uint16_t*>(W_g), draft, logp_joint,
+                     nullptr, nullptr, nullptr, logp_prefix, static_cast<uint8_t*>(workspace), L, dev_status,
+                     di->sms, reinterpret_cast<cudaStream_t>(stream));
+}
+
+int cpmtp_forward_host(const cpmtp_shape* shape, const void* h_host, const void* W_head, const void* E,
+                       const void* W_g, const int32_t* x_host, float* logp_host, float* loss_host,
+                       const cpmtp_saved* saved, void* workspace, size_t workspace_bytes, int32_t* dev_status,
+                       cpmtp_stream stream) {
+  if (validate_shape(shape) != CPMTP_OK) return validate_shape(shape);
+  if (!h_host || !x_host || !workspace) return CPMTP_ERR_NULL;
+  if (!aligned(workspace, kAlign)) return CPMTP_ERR_ALIGN;
+  const size_t fwd_bytes = cpmtp_workspace_bytes(shape, CPMTP_OP_FORWARD);
+  if (workspace_bytes < fwd_bytes + cpmtp_host_staging_bytes(shape)) return CPMTP_ERR_WORKSPACE;
+  cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
+  uint8_t* stage = static_cast<uint8_t*>(workspace) + align_up(fwd_bytes);
+  const size_t h_bytes = 2ull * shape->N * shape->d, x_bytes = 4ull * shape->N * shape->n;
+  uint8_t* h_dev = stage;
+  uint8_t* x_dev = h_dev + align_up(h_bytes);
+  uint8_t* logp_dev = x_dev + align_up(x_bytes);
+  uint8_t* loss_dev = logp_dev + align_up(4ull * shape->N);
+  CPMTP_TRY(cudaMemcpyAsync(h_dev, h_host, h_bytes, cudaMemcpyHostToDevice, st));
+  CPMTP_TRY(cudaMemcpyAsync(x_dev, x_host, x_bytes, cudaMemcpyHostToDevice, st));
+  const int rc = cpmtp_forward(shape, h_dev, W_head, E, W_g, reinterpret_cast<const int32_t*>(x_dev),
+                               reinterpret_cast<float*>(logp_dev), reinterpret_cast<float*>(loss_dev), saved,
+                               nullptr, workspace, fwd_bytes, dev_status, stream);
+  if (rc != CPMTP_OK) return rc;
+  if (logp_host != nullptr)
+    CPMTP_TRY(cudaMemcpyAsync(logp_host, logp_dev, 4ull * shape->N, cudaMemcpyDeviceToHost, st));
+  if (loss_host != nullptr) CPMTP_TRY(cudaMemcpyAsync(loss_host, loss_dev, 4, cudaMemcpyDeviceToHost, st));
+  return CPMTP_OK;
+}
+
+int cpmtp_backward(const cpmtp_shape* shape, const void* h, const void* W_head, const void* E, const void* W_g,
+                   const int32_t* x, const cpmtp_saved* saved, const float* dloss_dlogp, void* dh, void* dW_head,
+                   void* dE, void* dW_g, void* workspace, size_t workspace_bytes, int32_t* dev_status,
+                   cpmtp_stream stream) {
+  DeviceInfo* di = nullptr;
+  const int rc = check_common(shape, h, W_head, E, W_g, x, workspace, &di);
+  if (rc != CPMTP_OK) return rc;
+  if (saved == nullptr || !dh || !dW_head || !dE || !dW_g) return CPMTP_ERR_NULL;
+  const int rs = check_saved(saved);
+  if (rs != CPMTP_OK) return rs;
+  if (!aligned(dh, 16) || !aligned(dW_head, 16) || !aligned(dE, 16) || !aligned(dW_g, 16)) return CPMTP_ERR_ALIGN;
+  const cpmtp_shape& s = *shape;
+  const BwdLayout L = bwd_layout(s);
+  if (workspace_bytes < L.total) return CPMTP_ERR_WORKSPACE;
+  cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
+  uint8_t* ws = static_cast<uint8_t*>(workspace);
+  float* coef = reinterpret_cast<float*>(ws + L.coef);
+  float* dg = reinterpret_cast<float*>(ws + L.dg);
+  uint16_t* dz = reinterpret_cast<uint16_t*>(ws + L.dz);
+  uint16_t* G = reinterpret_cast<uint16_t*>(ws + L.G);
+  float* dE32 = reinterpret_cast<float*>(ws + L.dE32);
+  float* dwg_part = reinterpret_cast<float*>(ws + L.dwg_part);
+  const uint16_t* z = static_cast<const uint16_t*>(saved->z);
+  const uint16_t* Eb = static_cast<const uint16_t*>(E);
+  const int sms = di->sms;
+  const int K = L.K, d = s.d, V = s.V;
+  const int ncols = K * d;
+  const float aux = (s.flags & CPMTP_FLAG_AUX) ? s.aux_coef : 0.f;
+
+  coeff_kernel<<<(s.N + 255) / 256, 256, 0, st>>>(saved->q, saved->logw, saved->wbar, dloss_dlogp, coef, dg, s.N,
+                                                 s.r, aux);
+  CPMTP_TRY(cudaGetLastError());
+
+  const int d_tiles = (d + kBN - 1) / kBN;
+  for (int c = 0; c < L.chunks; ++c) {
+    const long long row0 = static_cast<long long>(c) * L.chunk_rows;
+    const int rows = static_cast<int>((L.M - row0) < L.chunk_rows ? (L.M - row0) : L.chunk_rows);
+    const uint16_t* zc = z + row0 * d;
+    const int m_tiles = (rows + kBM - 1) / kBM;
+    // recompute logits tile by tile -> G = dloss/dS (bf16), never more than one chunk
+    {
+      EpiLogitGrad<kBN>::Params ep{G, saved->lse, coef, x, row0, rows, L.ldg, V, K, s.n, s.r};
+      const int n_tiles = (L.ldg + kBN - 1) / kBN;
+      const Sched sc = make_sched(m_tiles, n_tiles, n_tiles, 16, d / kBK);
+      CPMTP_TRY((launch_gemm<CfgKK, EpiLogitGrad<kBN>>(zc, rows, d, Eb, V, d, d, sc, ep, dev_status, sms, st)));
+    }
+    // dz[rows, d] = G[rows, V] * E[V, d]
+    {
+      EpiStoreBf16<kBN, false>::Params ep{dz + row0 * d, nullptr, nullptr, rows, d, d, 0};
+      const Sched sc = make_sched(m_tiles, d_tiles, d_tiles, 16, (V + kBK - 1) / kBK);
+      CPMTP_TRY((launch_gemm<CfgKM, EpiStoreBf16<kBN, false>>(G, rows, L.ldg, Eb, d, d, V, sc, ep, dev_status, sms, st)));
+    }
+    // dE[V, d] (+)= G^T[V, rows] * z[rows, d]
+    {
+      const int v_tiles = (V + kBM - 1) / kBM;
+      const Sched sc = make_sched(v_tiles, d_tiles, d_tiles, 16, (rows + kBK - 1) / kBK);
+      if (L.chunks == 1) {
+        EpiStoreBf16<kBN, false>::Params ep{static_cast<uint16_t*>(dE), nullptr, nullptr, V, d, d, 0};
+        CPMTP_TRY((launch_gemm<CfgMM, EpiStoreBf16<kBN, false>>(G, V, L.ldg, zc, d, d, rows, sc, ep, dev_status, sms, st)));
+      } else {
+        EpiAccumF32<kBN>::Params ep{dE32, V, d, d, c > 0 ? 1 : 0};
+        CPMTP_TRY((launch_gemm<CfgMM, EpiAccumF32<kBN>>(G, V, L.ldg, zc, d, d, rows, sc, ep, dev_status, sms, st)));
+      }
+    }
+  }
+  if (L.chunks > 1) {
+    f32_to_bf16_kernel<<<sms * 8, 256, 0, st>>>(dE32, static_cast<uint16_t*>(dE), static_cast<size_t>(V) * d);
+    CPMTP_TRY(cudaGetLastError());
+  }
+  // dW_head[K*d, d] = dz^T[K*d, N] * h[N, d]
+  {
+    EpiStoreBf16<kBN, false>::Params ep{static_cast<uint16_t*>(dW_head), nullptr, nullptr, ncols, d, d, 0};
+    const int m_tiles = (ncols + kBM - 1) / kBM;
+    const Sched sc = make_sched(m_tiles, d_tiles, d_tiles, 16, (s.N + kBK - 1) / kBK);
+    CPMTP_TRY((launch_gemm<CfgMM, EpiStoreBf16<kBN, false>>(dz, ncols, ncols, h, d, d, s.N, sc, ep, dev_status, sms, st)));
+  }
+  // dh[N, d] = dz[N, K*d] * W_cat[K*d, d] + dg * W_g
+  {
+    EpiStoreBf16<kBN, true>::Params ep{static_cast<uint16_t*>(dh), dg, static_cast<const uint16_t*>(W_g), s.N, d, d, s.r};
+    const int m_tiles = (s.N + kBM - 1) / kBM;
+    const Sched sc = make_sched(m_tiles, d_tiles, d_tiles, 16, ncols / kBK);
+    CPMTP_TRY((launch_gemm<CfgKM, EpiStoreBf16<kBN, true>>(dz, s.N, ncols, W_head, d, d, ncols, sc, ep, dev_status, sms, st)));
+  }
+  // dW_g[r, d] = dg^T * h
+  {
+    dim3 grid((d + 127) / 128, L.dwg_slices);
+    dwg_partial_kernel<CPMTP_MAX_R><<<grid, 128, 0, st>>>(dg, static_cast<const uint16_t*>(h), dwg_part, s.N, d, s.r,
+                                                          L.dwg_rows_per_slice);
+    CPMTP_TRY(cudaGetLastError());
+    dwg_reduce_kernel<<<(s.r * d + 255) / 256, 256, 0, st>>>(dwg_part, static_cast<uint16_t*>(dW_g), L.dwg_slices,
+                                                            s.r, d);
+    CPMTP_TRY(cudaGetLastError());
+  }
+  return CPMTP_OK;
+}
+
+}  // extern "C"

@@ -1,0 +1,227 @@
+// The O(N*r) and O(N*r*d) stages around the tensor-core GEMMs: gate, mixture
+// epilogue, loss, backward coefficients, gate-weight gradient, dtype conversion.
+// All reductions run in a fixed order (no floating-point atomics) so results are
+// reproducible from run to run.
+#pragma once
+#include <cstdint>
+
+#include "ptx.cuh"
+
+namespace cpmtp {
+
+__device__ __forceinline__ float warp_sum(float v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+  return v;
+}
+__device__ __forceinline__ float warp_max(float v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, o));
+  return v;
+}
+
+// Gate of Eq. 7: logw[i, :] = log softmax(W_g h[i]).  One warp per position,
+// lane a ends up holding expert a (r <= 32).
+__global__ void gate_kernel(const uint16_t* __restrict__ h, const uint16_t* __restrict__ W_g,
+                            float* __restrict__ logw, int N, int d, int r) {
+  const int warps_per_block = blockDim.x >> 5;
+  const int i = blockIdx.x * warps_per_block + (threadIdx.x >> 5);
+  const int lane = threadIdx.x & 31;
+  if (i >= N) return;
+  const uint4* hrow = reinterpret_cast<const uint4*>(h + static_cast<size_t>(i) * d);
+  const int vecs = d >> 3;
+  float mine = -INFINITY;
+  for (int a = 0; a < r; ++a) {
+    const uint4* wrow = reinterpret_cast<const uint4*>(W_g + static_cast<size_t>(a) * d);
+    float acc = 0.f;
+    for (int j = lane; j < vecs; j += 32) {
+      const uint4 hv = __ldg(hrow + j);
+      const uint4 wv = __ldg(wrow + j);
+      acc = fmaf(ptx::bf16_lo(hv.x), ptx::bf16_lo(wv.x), acc);
+      acc = fmaf(ptx::bf16_hi(hv.x), ptx::bf16_hi(wv.x), acc);
+      acc = fmaf(ptx::bf16_lo(hv.y), ptx::bf16_lo(wv.y), acc);
+      acc = fmaf(ptx::bf16_hi(hv.y), ptx::bf16_hi(wv.y), acc);
+      acc = fmaf(ptx::bf16_lo(hv.z), ptx::bf16_lo(wv.z), acc);
+      acc = fmaf(ptx::bf16_hi(hv.z), ptx::bf16_hi(wv.z), acc);
+      acc = fmaf(ptx::bf16_lo(hv.w), ptx::bf16_lo(wv.w), acc);
+      acc = fmaf(ptx::bf16_hi(hv.w), ptx::bf16_hi(wv.w), acc);
+    }
+    acc = warp_sum(acc);
+    if (lane == a) mine = acc;
+  }
+  const float m = warp_max(mine);
+  const float e = lane < r ? expf(mine - m) : 0.f;
+  const float lse = m + logf(warp_sum(e));
+  if (lane < r) logw[static_cast<size_t>(i) * r + lane] = mine - lse;
+}
+
+// Mixture epilogue (last line of Eq. 9).  One warp per position.
+//   lse[i,k]  = two-pass merge of the per-split (max, sum-exp) partials
+//   tgt[i,k]  = sum of the per-64-column target-logit partials
+//   a[i,al]   = logw[i,al] + sum_s (tgt - lse)[i, s*r+al]
+//   logp[i]   = logsumexp_al a;  q = exp(a - logp)
+// Optionally the prefix scores logsumexp_al(logw + sum_{t<=s} C) for every s.
+__global__ void mixture_kernel(const float* __restrict__ part_m, const float* __restrict__ part_l,
+                               int splits, const float* __restrict__ tgt_part, int tgt_parts,
+                               const float* __restrict__ logw, float* __restrict__ lse_out,
+                               float* __restrict__ tgt_out, float* __restrict__ q_out,
+                               float* __restrict__ logp, float* __restrict__ logp_prefix, int N, int n,
+                               int r) {
+  const int warps_per_block = blockDim.x >> 5;
+  const int i = blockIdx.x * warps_per_block + (threadIdx.x >> 5);
+  const int lane = threadIdx.x & 31;
+  if (i >= N) return;
+  const int K = n * r;
+  float a = lane < r ? logw[static_cast<size_t>(i) * r + lane] : -INFINITY;
+  for (int s = 0; s < n; ++s) {
+    for (int al = 0; al < r; ++al) {
+      const int k = s * r + al;
+      const size_t row = static_cast<size_t>(i) * K + k;
+      // pass 1: global max over splits; pass 2: rescaled sum
+      float m = -INFINITY;
+      for (int j = lane; j < splits; j += 32) m = fmaxf(m, part_m[row * splits + j]);
+      m = warp_max(m);
+      float l = 0.f;
+      for (int j = lane; j < splits; j += 32)
+        l += part_l[row * splits + j] * exp2f(part_m[row * splits + j] - m);
+      l = warp_sum(l);
+      const float lse = (m + log2f(l)) * 0.6931471805599453f;
+      float t = 0.f;
+      for (int j = lane; j < tgt_parts; j += 32) t += tgt_part[row * tgt_parts + j];
+      t = warp_sum(t);
+      if (lane == al) {
+        a += t - lse;
+        if (lse_out != nullptr) lse_out[row] = lse;
+        if (tgt_out != nullptr) tgt_out[row] = t;
+      }
+    }
+    if (logp_prefix != nullptr || s == n - 1) {
+      const float m = warp_max(a);
+      const float e = lane < r ? expf(a - m) : 0.f;
+      const float lp = m + logf(warp_sum(e));
+      if (logp_prefix != nullptr && lane == 0) logp_prefix[static_cast<size_t>(i) * n + s] = lp;
+      if (s == n - 1) {
+        if (lane == 0) logp[i] = lp;
+        if (q_out != nullptr && lane < r) q_out[static_cast<size_t>(i) * r + lane] = expf(a - lp);
+      }
+    }
+  }
+}
+
+// Loss, mean gate weights and hard expert counts (Eq. 10's n_a).  One block.
+//   wbar[a] = (1/N) sum_i exp(logw[i,a]);  counts[a] = #{i : argmax_b w[i,b] = a}
+//   loss = -(1/N) sum_i logp[i] + aux_coef * sum_a wbar[a]^2
+__global__ void finalize_kernel(const float* __restrict__ logp, const float* __restrict__ logw,
+                                float* __restrict__ wbar, int* __restrict__ counts,
+                                float* __restrict__ loss, int N, int r, float aux_coef) {
+  __shared__ double red[1024];
+  __shared__ int redi[1024];
+  __shared__ double wbar_s[32];
+  const int t = threadIdx.x;
+  for (int a = 0; a <= r; ++a) {   // a == r: the logp sum
+    double acc = 0.0;
+    int cnt = 0;
+    for (int i = t; i < N; i += blockDim.x) {
+      if (a < r) {
+        const float* row = logw + static_cast<size_t>(i) * r;
+        acc += static_cast<double>(expf(row[a]));
+        bool is_max = true;
+        for (int b = 0; b < r; ++b)
+          if (row[b] > row[a] || (row[b] == row[a] && b < a)) is_max = false;
+        cnt += is_max ? 1 : 0;
+      } else {
+        acc += static_cast<double>(logp[i]);
+      }
+    }
+    red[t] = acc;
+    redi[t] = cnt;
+    __syncthreads();
+    for (int o = blockDim.x >> 1; o > 0; o >>= 1) {
+      if (t < o) {
+        red[t] += red[t + o];
+        redi[t] += redi[t + o];
+      }
+      __syncthreads();
+    }
+    if (t == 0) {
+      if (a < r) {
+        wbar_s[a] = red[0] / N;
+        if (wbar != nullptr) wbar[a] = static_cast<float>(wbar_s[a]);
+        if (counts != nullptr) counts[a] = redi[0];
+      } else if (loss != nullptr) {
+        double aux = 0.0;
+        for (int b = 0; b < r; ++b) aux += wbar_s[b] * wbar_s[b];
+        *loss = static_cast<float>(-red[0] / N + static_cast<double>(aux_coef) * aux);
+      }
+    }
+    __syncthreads();
+  }
+}
+
+// Backward coefficients (derivative of Eq. 9 and of the gate softmax of Eq. 7).
+//   c[i,a]  = up_i * q[i,a]
+//   dg[i,b] = up_i * (q[i,b] - w[i,b]) + w[i,b] * (u_b - sum_g w[i,g] u_g),  u_b = 2 aux wbar_b / N
+__global__ void coeff_kernel(const float* __restrict__ q, const float* __restrict__ logw,
+                             const float* __restrict__ wbar, const float* __restrict__ up,
+                             float* __restrict__ coef, float* __restrict__ dg, int N, int r,
+                             float aux_coef) {
+  const int i = blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= N) return;
+  const float u_i = up != nullptr ? up[i] : -1.0f / N;
+  const float scale = 2.0f * aux_coef / N;
+  float wu = 0.f;
+  for (int b = 0; b < r; ++b) wu += expf(logw[static_cast<size_t>(i) * r + b]) * scale * wbar[b];
+  for (int b = 0; b < r; ++b) {
+    const float w = expf(logw[static_cast<size_t>(i) * r + b]);
+    const float qq = q[static_cast<size_t>(i) * r + b];
+    coef[static_cast<size_t>(i) * r + b] = u_i * qq;
+    dg[static_cast<size_t>(i) * r + b] = u_i * (qq - w) + w * (scale * wbar[b] - wu);
+  }
+}
+
+// dW_g[b, :] = sum_i dg[i, b] * h[i, :]  in two deterministic stages.
+// Stage 1: block (column chunk, position slice) -> part[slice, b, col].
+template <int R_MAX>
+__global__ void dwg_partial_kernel(const float* __restrict__ dg, const uint16_t* __restrict__ h,
+                                   float* __restrict__ part, int N, int d, int r, int rows_per_slice) {
+  const int col = blockIdx.x * blockDim.x + threadIdx.x;
+  const int slice = blockIdx.y;
+  if (col >= d) return;
+  float acc[R_MAX];
+#pragma unroll
+  for (int b = 0; b < R_MAX; ++b) acc[b] = 0.f;
+  const int i0 = slice * rows_per_slice;
+  const int i1 = min(N, i0 + rows_per_slice);
+  for (int i = i0; i < i1; ++i) {
+    const float hv = __uint_as_float(static_cast<uint32_t>(h[static_cast<size_t>(i) * d + col]) << 16);
+    const float* g = dg + static_cast<size_t>(i) * r;
+#pragma unroll
+    for (int b = 0; b < R_MAX; ++b)
+      if (b < r) acc[b] = fmaf(g[b], hv, acc[b]);
+  }
+#pragma unroll
+  for (int b = 0; b < R_MAX; ++b)
+    if (b < r) part[(static_cast<size_t>(slice) * r + b) * d + col] = acc[b];
+}
+// Stage 2: sum the slices in order and round to bf16.
+__global__ void dwg_reduce_kernel(const float* __restrict__ part, uint16_t* __restrict__ dW_g, int slices,
+                                  int r, int d) {
+  const int idx = blockIdx.x * blockDim.x + threadIdx.x;
+  if (idx >= r * d) return;
+  float acc = 0.f;
+  for (int s = 0; s < slices; ++s) acc += part[static_cast<size_t>(s) * r * d + idx];
+  dW_g[idx] = static_cast<uint16_t>(ptx::pack_bf16x2(acc, 0.f) & 0xFFFFu);
+}
+
+__global__ void f32_to_bf16_kernel(const float* __restrict__ src, uint16_t* __restrict__ dst, size_t count) {
+  const size_t stride = static_cast<size_t>(gridDim.x) * blockDim.x * 4;
+  for (size_t i = (static_cast<size_t>(blockIdx.x) * blockDim.x + threadIdx.x) * 4; i < count; i += stride) {
+    const float4 v = *reinterpret_cast<const float4*>(src + i);
+    uint2 o;
+    o.x = ptx::pack_bf16x2(v.x, v.y);
+    o.y = ptx::pack_bf16x2(v.z, v.w);
+    *reinterpret_cast<uint2*>(dst + i) = o;
+  }
+}
+
+}  // namespace cpmtp
