@@ -1,0 +1,179 @@
+"""GPU parity: the CUDA library (through its C-ABI) against the fp64 oracle on the
+same seeded bf16 inputs.  Tolerances: |delta log P| <= 2e-3 per position, gradient
+relative L2 error <= 1e-2."""
+import os
+
+import numpy as np
+import pytest
+import torch
+
+from oracle import cp_head
+from paper_2410_17765_b200 import synth
+
+pytestmark = pytest.mark.gpu
+
+LOGP_TOL = 2e-3
+GRAD_TOL = 1e-2
+
+
+def to_dev(inp):
+    return [t.cuda() for t in (inp.h, inp.W_head, inp.E, inp.W_g, inp.x)]
+
+
+def rel_l2(a, b):
+    a = np.asarray(a, dtype=np.float64)
+    b = np.asarray(b, dtype=np.float64)
+    return float(np.linalg.norm(a - b) / max(np.linalg.norm(b), 1e-300))
+
+
+def status_tensor():
+    return torch.zeros(1, dtype=torch.int32, device="cuda")
+
+
+CASES = {
+    "tiny": dict(shape=synth.CONFIGS["tiny"]),
+    "ragged": dict(shape=synth.Shape(N=70, d=320, V=1000, n=2, r=3)),
+    "ragged_stress": dict(shape=synth.Shape(N=37, d=192, V=777, n=3, r=5), weight_scale=8.0),
+    "rank1": dict(shape=synth.Shape(N=130, d=128, V=300, n=4, r=1)),
+    "wide": dict(shape=synth.Shape(N=300, d=512, V=2100, n=2, r=8), targets="zipf"),
+}
+
+
+@pytest.mark.parametrize("name", list(CASES))
+def test_forward_matches_oracle(name):
+    from paper_2410_17765_b200 import binding
+
+    kw = dict(CASES[name])
+    shape = kw.pop("shape")
+    inp = synth.make_inputs(shape, seed=0, **kw)
+    ref = cp_head.forward(inp.h, inp.W_head, inp.E, inp.W_g, inp.x, shape.n, shape.r, aux_coef=1.0)
+    st = status_tensor()
+    saved = binding.Saved.alloc(binding.make_shape(shape.N, shape.d, shape.V, shape.n, shape.r))
+    out = binding.forward(*to_dev(inp), aux_coef=1.0, saved=saved, want_counts=True, dev_status=st)
+    torch.cuda.synchronize()
+    assert int(st.item()) == 0
+    logp = out["logp"].cpu().numpy()
+    assert np.max(np.abs(logp - ref.logp)) <= LOGP_TOL
+    assert abs(float(out["loss"].item()) - ref.loss) <= LOGP_TOL
+    assert np.max(np.abs(saved.lse.cpu().numpy() - ref.lse)) <= 1e-3
+    assert np.max(np.abs(saved.tgt.cpu().numpy() - ref.tgt)) <= 1e-3 * max(1.0, np.abs(ref.tgt).max())
+    assert np.max(np.abs(saved.q.cpu().numpy() - ref.q)) <= 2e-3
+    assert np.max(np.abs(saved.logw.cpu().numpy() - ref.logw)) <= 1e-4
+    assert np.max(np.abs(saved.wbar[: shape.r].cpu().numpy() - ref.wbar)) <= 1e-5
+    assert out["counts"].cpu().numpy().sum() == shape.N
+
+
+@pytest.mark.parametrize("name,chunk_rows", [("tiny", None), ("tiny", 256), ("ragged", 128), ("ragged_stress", None),
+                                             ("rank1", None), ("wide", 1024)])
+def test_backward_matches_oracle(name, chunk_rows):
+    from paper_2410_17765_b200 import binding
+
+    kw = dict(CASES[name])
+    shape = kw.pop("shape")
+    inp = synth.make_inputs(shape, seed=0, **kw)
+    ref = cp_head.backward(inp.h, inp.W_head, inp.E, inp.W_g, inp.x, shape.n, shape.r, aux_coef=1.0)
+    dev = to_dev(inp)
+    saved = binding.Saved.alloc(binding.make_shape(shape.N, shape.d, shape.V, shape.n, shape.r))
+    st = status_tensor()
+    old = os.environ.get("CPMTP_BWD_CHUNK_ROWS")
+    try:
+        if chunk_rows is not None:
+            os.environ["CPMTP_BWD_CHUNK_ROWS"] = str(chunk_rows)
+        binding.forward(*dev, aux_coef=1.0, saved=saved, dev_status=st)
+        g = binding.backward(*dev, saved, aux_coef=1.0, dev_status=st)
+        torch.cuda.synchronize()
+    finally:
+        if old is None:
+            os.environ.pop("CPMTP_BWD_CHUNK_ROWS", None)
+        else:
+            os.environ["CPMTP_BWD_CHUNK_ROWS"] = old
+    assert int(st.item()) == 0
+    for key, want in (("dh", ref.dh), ("dW_head", ref.dW_head), ("dE", ref.dE), ("dW_g", ref.dW_g)):
+        got = g[key].float().cpu().numpy()
+        if np.linalg.norm(want) == 0:
+            assert np.abs(got).max() == 0, key
+        else:
+            assert rel_l2(got, want) <= GRAD_TOL, (key, rel_l2(got, want))
+
+
+def test_backward_with_upstream_gradient():
+    from paper_2410_17765_b200 import binding
+
+    shape = CASES["ragged"]["shape"]
+    inp = synth.make_inputs(shape, seed=3)
+    up = torch.linspace(-1.0, 0.5, shape.N, dtype=torch.float32)
+    ref = cp_head.backward(inp.h, inp.W_head, inp.E, inp.W_g, inp.x, shape.n, shape.r, dloss_dlogp=up.numpy())
+    dev = to_dev(inp)
+    saved = binding.Saved.alloc(binding.make_shape(shape.N, shape.d, shape.V, shape.n, shape.r))
+    binding.forward(*dev, saved=saved)
+    g = binding.backward(*dev, saved, dloss_dlogp=up.cuda())
+    torch.cuda.synchronize()
+    for key, want in (("dh", ref.dh), ("dW_head", ref.dW_head), ("dE", ref.dE), ("dW_g", ref.dW_g)):
+        assert rel_l2(g[key].float().cpu().numpy(), want) <= GRAD_TOL, key
+
+
+@pytest.mark.parametrize("N", [1, 8, 64])
+def test_score_draft_matches_oracle(N):
+    from paper_2410_17765_b200 import binding
+
+    shape = synth.Shape(N=N, d=256, V=5000, n=4, r=8)
+    inp = synth.make_inputs(shape, seed=N)
+    ref = cp_head.forward(inp.h, inp.W_head, inp.E, inp.W_g, inp.x, shape.n, shape.r)
+    pre = cp_head.prefix_log_probs(ref)
+    st = status_tensor()
+    out = binding.score_draft(*to_dev(inp), dev_status=st)
+    torch.cuda.synchronize()
+    assert int(st.item()) == 0
+    assert np.max(np.abs(out["logp_joint"].cpu().numpy() - ref.logp)) <= LOGP_TOL
+    assert np.max(np.abs(out["logp_prefix"].cpu().numpy() - pre)) <= LOGP_TOL
+
+
+def test_out_of_range_target_is_clamped_and_reported():
+    from paper_2410_17765_b200 import binding
+
+    shape = synth.Shape(N=16, d=128, V=100, n=2, r=2)
+    inp = synth.make_inputs(shape, seed=1)
+    bad = inp.x.clone()
+    bad[3, 1] = shape.V + 5
+    clamped = inp.x.clone()
+    clamped[3, 1] = shape.V - 1
+    ref = cp_head.forward(inp.h, inp.W_head, inp.E, inp.W_g, clamped, shape.n, shape.r)
+    st = status_tensor()
+    h, W, E, Wg, _ = to_dev(inp)
+    out = binding.forward(h, W, E, Wg, bad.cuda(), dev_status=st)
+    torch.cuda.synchronize()
+    assert int(st.item()) == 1
+    assert np.max(np.abs(out["logp"].cpu().numpy() - ref.logp)) <= LOGP_TOL
+
+
+def test_run_to_run_determinism():
+    from paper_2410_17765_b200 import binding
+
+    shape = CASES["wide"]["shape"]
+    inp = synth.make_inputs(shape, seed=0)
+    dev = to_dev(inp)
+    cs = binding.make_shape(shape.N, shape.d, shape.V, shape.n, shape.r)
+    outs = []
+    for _ in range(2):
+        saved = binding.Saved.alloc(cs)
+        f = binding.forward(*dev, saved=saved)
+        g = binding.backward(*dev, saved)
+        torch.cuda.synchronize()
+        outs.append((f["logp"].clone(), g["dE"].clone(), g["dh"].clone(), g["dW_head"].clone()))
+    for a, b in zip(*outs):
+        assert torch.equal(a, b)
+
+
+def test_forward_host_matches_device_forward():
+    from paper_2410_17765_b200 import binding
+
+    shape = CASES["tiny"]["shape"]
+    inp = synth.make_inputs(shape, seed=0)
+    h, W, E, Wg, x = to_dev(inp)
+    want = binding.forward(h, W, E, Wg, x)
+    logp_host = torch.empty(shape.N, dtype=torch.float32).pin_memory()
+    loss_host = torch.empty(1, dtype=torch.float32).pin_memory()
+    binding.forward_host(inp.h.pin_memory(), W, E, Wg, inp.x.pin_memory(), logp_host, loss_host)
+    torch.cuda.synchronize()
+    assert torch.equal(logp_host, want["logp"].cpu())
+    assert torch.equal(loss_host, want["loss"].cpu())
