@@ -1,0 +1,325 @@
+#!/usr/bin/env python
+"""Benchmark of the fused CP-head log-likelihood on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload NAME] [--impl ours|reference]
+
+One step = one pass of the whole path of the workload over one batch of seeded
+synthetic inputs: forward for `train_fwd`, forward + backward for the `*_fwd_bwd`
+workloads, draft scoring for `decode_*`.  Prints ONE JSON line.  With N > 1 ranks
+(torchrun) every rank runs the same per-GPU batch (positions are independent, no
+collective on the data path) and the reported value is the whole-job rate.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "cp_head_positions_per_second"
+UNIT = "positions/s"
+
+WORKLOADS = {
+    # name: (synth config, kind, extra make_inputs kwargs, aux coefficient)
+    "train_fwd": ("train_fwd", "fwd", {}, None),
+    "train_fwd_bwd": ("train_fwd_bwd", "fwd_bwd", {}, None),
+    "bigvocab_fwd_bwd": ("bigvocab_fwd_bwd", "fwd_bwd", {"targets": "zipf"}, 1.0),
+    "decode_1": ("decode_1", "score", {}, None),
+    "decode_8": ("decode_8", "score", {}, None),
+    "decode_64": ("decode_64", "score", {}, None),
+    "tiny": ("tiny", "fwd_bwd", {}, None),
+}
+
+# dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel, from the ncu
+# captures summarised under profiles/ (None until captured, or once the kernel has changed since).
+NCU_TRAFFIC_BYTES = {}
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            p = json.load(f)
+        return dict(hbm_gbs=p["hbm_gbs"], burst=p["bf16_tflops"], sustained=p["bf16_tflops_sustained"], src="measured")
+    return dict(hbm_gbs=6650.0, burst=1590.0, sustained=1400.0, src="fallback")
+
+
+class ClockSampler:
+    """nvidia-smi clock / throttle-reason samples taken while the timed region runs."""
+
+    FIELDS = ("clocks.sm,clocks.max.sm,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+              "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index: int):
+        self.proc = None
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--id={gpu_index}", f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits",
+                 "-lms", "100"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+        except OSError:
+            self.proc = None
+
+    def stop(self) -> dict:
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            out, _ = self.proc.communicate(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+            out, _ = self.proc.communicate()
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for line in out.strip().splitlines():
+            parts = [p.strip() for p in line.split(",")]
+            if len(parts) < 6:
+                continue
+            try:
+                sm.append(float(parts[0]))
+                mx.append(float(parts[1]))
+            except ValueError:
+                continue
+            for name, val in zip(names, parts[2:6]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "samples": len(sm), "reasons": sorted(reasons)}
+
+
+def flops_per_position(s, kind):
+    K = s.n * s.r
+    fwd = 2 * K * (s.d * s.d + s.V * s.d) + 2 * s.r * s.d
+    return fwd if kind != "fwd_bwd" else 3 * fwd
+
+
+def oracle_seconds_per_position(inp, kind, aux, sample: int):
+    """Time the fp64 oracle, as it stands, on the first `sample` positions."""
+    import torch
+    from oracle import cp_head
+    from paper_2410_17765_b200 import synth
+
+    s = inp.shape
+    sample = min(sample, s.N)
+    sub = synth.subsample_positions(inp, torch.arange(sample))
+    t0 = time.perf_counter()
+    if kind == "fwd_bwd":
+        cp_head.backward(sub.h, sub.W_head, sub.E, sub.W_g, sub.x, s.n, s.r, aux_coef=aux or 0.0)
+    else:
+        cp_head.forward(sub.h, sub.W_head, sub.E, sub.W_g, sub.x, s.n, s.r, aux_coef=aux or 0.0)
+    return (time.perf_counter() - t0) / sample, sample
+
+
+def blas_threads() -> int:
+    try:
+        from threadpoolctl import threadpool_info
+
+        counts = [p.get("num_threads", 1) for p in threadpool_info() if p.get("user_api") == "blas"]
+        if counts:
+            return max(counts)
+    except Exception:
+        pass
+    return len(os.sched_getaffinity(0))
+
+
+def oracle_sample_size(s, kind) -> int:
+    # about 10-30 s of fp64 numpy work: assume ~40 GFLOP/s on the host cores
+    per_pos = flops_per_position(s, kind) * (1.4 if kind == "fwd_bwd" else 1.0)
+    return max(1, min(s.N, int(40e9 * 15 / per_pos)))
+
+
+def run_reference(args, rank: int):
+    """--impl reference: the oracle, as it stands, on the host cores (rank 0 only)."""
+    if rank != 0:
+        return
+    from paper_2410_17765_b200 import synth
+
+    cfg, kind, extra, aux = WORKLOADS[args.workload]
+    shape = synth.CONFIGS[cfg]
+    inp = synth.make_inputs(shape, seed=0, **extra)
+    # bounded sample per step so that the whole run ends within a few minutes
+    per_step = max(1, oracle_sample_size(shape, kind) // max(1, 2 * (args.steps + args.warmup)))
+    for _ in range(args.warmup):
+        oracle_seconds_per_position(inp, kind, aux, per_step)
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        oracle_seconds_per_position(inp, kind, aux, per_step)
+    dt = time.perf_counter() - t0
+    value = per_step * args.steps / dt
+    cores = blas_threads()
+    sample = f"first {per_step} of {shape.N} positions per step at full d, V, n, r"
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": 1e3 * dt / args.steps, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": args.workload, "kind": kind, **shape.__dict__},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line))
+
+
+def run_ours(args, rank: int, world: int, local_rank: int):
+    import torch
+
+    from paper_2410_17765_b200 import binding, synth
+
+    if not torch.cuda.is_available():
+        raise RuntimeError("bench.py needs a CUDA device; there is no CPU fallback")
+    torch.cuda.set_device(local_rank)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist_mod
+
+        dist = dist_mod
+        dist.init_process_group(backend="nccl", device_id=torch.device("cuda", local_rank))
+
+    cfg, kind, extra, aux = WORKLOADS[args.workload]
+    shape = synth.CONFIGS[cfg]
+    inp = synth.make_inputs(shape, seed=rank, **extra)
+    h, W_head, E, W_g, x = [t.cuda() for t in (inp.h, inp.W_head, inp.E, inp.W_g, inp.x)]
+    cs = binding.make_shape(shape.N, shape.d, shape.V, shape.n, shape.r, aux)
+    ws_fwd = binding.alloc_workspace(binding.workspace_bytes(cs, binding.OP_FORWARD) +
+                                     binding.host_staging_bytes(cs) + 512)
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    saved = binding.Saved.alloc(cs) if kind == "fwd_bwd" else None
+    ws_bwd = binding.alloc_workspace(binding.workspace_bytes(cs, binding.OP_BACKWARD)) if kind == "fwd_bwd" else None
+    out_f, out_b, out_s = {}, {}, {}
+
+    def step():
+        if kind == "fwd":
+            binding.forward(h, W_head, E, W_g, x, aux_coef=aux, workspace=ws_fwd, dev_status=status, out=out_f)
+        elif kind == "fwd_bwd":
+            binding.forward(h, W_head, E, W_g, x, aux_coef=aux, saved=saved, workspace=ws_fwd, dev_status=status,
+                            out=out_f)
+            binding.backward(h, W_head, E, W_g, x, saved, aux_coef=aux, workspace=ws_bwd, dev_status=status,
+                             out=out_b)
+        else:
+            binding.score_draft(h, W_head, E, W_g, x, workspace=ws_fwd, dev_status=status, out=out_s)
+
+    h_pin, x_pin = inp.h.pin_memory(), inp.x.pin_memory()
+    logp_pin = torch.empty(shape.N, dtype=torch.float32).pin_memory()
+    loss_pin = torch.empty(1, dtype=torch.float32).pin_memory()
+
+    def step_e2e():
+        binding.forward_host(h_pin, W_head, E, W_g, x_pin, logp_pin, loss_pin, aux_coef=aux, saved=saved,
+                             workspace=ws_fwd, dev_status=status)
+        if kind == "fwd_bwd":
+            binding.backward(h, W_head, E, W_g, x, saved, aux_coef=aux, workspace=ws_bwd, dev_status=status,
+                             out=out_b)
+        torch.cuda.current_stream().synchronize()   # the step's result is read on the host
+
+    def barrier():
+        torch.cuda.synchronize()
+        if dist is not None:
+            dist.barrier()
+            torch.cuda.synchronize()
+
+    def timed(fn, steps, profile):
+        barrier()
+        if profile:
+            binding.profile_begin()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(steps):
+            fn()
+        e1.record()
+        torch.cuda.synchronize()
+        stages = binding.profile_end() if profile else {}
+        ms = e0.elapsed_time(e1)
+        barrier()
+        if dist is not None:
+            t = torch.tensor([ms], device="cuda", dtype=torch.float64)
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            ms = float(t.item())
+        return ms, stages
+
+    for _ in range(args.warmup):
+        step()
+    sampler = ClockSampler(local_rank) if rank == 0 else None
+    ms_total, stages = timed(step, args.steps, True)
+    clocks = sampler.stop() if sampler is not None else None
+    for _ in range(min(args.warmup, 3)):
+        step_e2e()
+    ms_e2e, _ = timed(step_e2e, args.steps, False)
+    if int(status.item()) != 0:
+        raise RuntimeError(f"device status {int(status.item())} raised during the benchmark")
+
+    if rank != 0:
+        if dist is not None:
+            dist.destroy_process_group()
+        return
+    peaks = measured_peaks()
+    positions = shape.N * world
+    value = positions * args.steps / (ms_total * 1e-3)
+    e2e_value = positions * args.steps / (ms_e2e * 1e-3)
+    K = shape.n * shape.r
+    dominant = "lse"
+    dom_ms, dom_launches = stages.get(dominant, (0.0, 0))
+    avg_ms = dom_ms / max(1, dom_launches)
+    if kind == "score" and shape.N * K * 2 < 250:   # below the ridge: HBM-bound streaming of E
+        alg = 2.0 * shape.V * shape.d
+        roof = {"bound": "hbm", "achieved": alg / (avg_ms * 1e-3) / 1e9, "peak": peaks["hbm_gbs"], "unit": "GB/s"}
+    else:
+        alg = 2.0 * shape.N * K * shape.V * shape.d
+        long_run = ms_total > 2000.0
+        roof = {"bound": "tensor", "achieved": alg / (avg_ms * 1e-3) / 1e12,
+                "peak": peaks["sustained"] if long_run else peaks["burst"], "unit": "TFLOP/s",
+                "peak_kind": "sustained" if long_run else "burst"}
+    roof["frac"] = roof["achieved"] / roof["peak"]
+    roof["traffic"] = NCU_TRAFFIC_BYTES.get(args.workload)
+    roof["kernel"] = "tc_gemm_kernel<EpiLse> (unembedding + logsumexp_V)"
+    roof["peak_source"] = peaks["src"]
+    roof["avg_launch_ms"] = avg_ms
+    roof["algorithmic_per_launch"] = alg
+    total_flops = flops_per_position(shape, kind) * positions * args.steps
+    n_sub = oracle_sample_size(shape, kind)
+    sec_per_pos, n_sub = oracle_seconds_per_position(inp, kind, aux, n_sub)
+    line = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+        "ms_per_step": ms_total / args.steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "bf16", "data": "synthetic",
+        "config": {"workload": args.workload, "kind": kind, **shape.__dict__, "aux_coef": aux,
+                   "targets": extra.get("targets", "uniform"), "l2": "inputs larger than L2 (no flush)",
+                   "per_gpu_positions": shape.N},
+        "clocks": clocks,
+        "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": shape.N * shape.d * 2 + shape.N * shape.n * 4,
+                "d2h_bytes_per_step": shape.N * 4 + 4, "ms_per_step": ms_e2e / args.steps},
+        "gpu_launches": int(sum(c for _, c in stages.values())),
+        "roofline": roof,
+        "cpu_baseline": {"value": 1.0 / sec_per_pos, "unit": UNIT, "cores": blas_threads(), "kind": "oracle",
+                         "sample": f"first {n_sub} of {shape.N} positions at full d, V, n, r (fp64 numpy)"},
+        "model_flops_tflops": total_flops / (ms_total * 1e-3) / 1e12,
+        "stages_ms_per_step": {k: v[0] / args.steps for k, v in stages.items()},
+    }
+    print(json.dumps(line))
+    if dist is not None:
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="train_fwd", choices=sorted(WORKLOADS))
+    args = ap.parse_args()
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    if args.impl == "reference":
+        run_reference(args, rank)
+    else:
+        run_ours(args, rank, world, local_rank)
+
+
+if __name__ == "__main__":
+    main()

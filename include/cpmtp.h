@@ -148,6 +148,36 @@ int cpmtp_forward_host(const cpmtp_shape* shape, const void* h_host, const void*
                        float* loss_host, const cpmtp_saved* saved, void* workspace,
                        size_t workspace_bytes, int32_t* dev_status, cpmtp_stream stream);
 
+/*
+ * Per-stage device timing, for benchmarks.  Between cpmtp_profile_begin() and
+ * cpmtp_profile_end() every kernel launch of the entry points above is bracketed
+ * by a pair of CUDA events on the launching stream (host-side bookkeeping only:
+ * the numerical path is unchanged).  cpmtp_profile_end() synchronises the device,
+ * writes the summed kernel time in milliseconds and the launch count of each
+ * stage into stage_ms[count] / stage_launches[count] (count <= CPMTP_STAGE_COUNT;
+ * either array may be NULL), releases the events and returns the total number of
+ * launches recorded, or a negative error code.  Not thread-safe; one device at a
+ * time.  The paper has no counterpart for these two calls.
+ */
+enum {
+  CPMTP_STAGE_GATE = 0,      /* Eq. 7 */
+  CPMTP_STAGE_PROJ,          /* head projection + target-logit partials */
+  CPMTP_STAGE_LSE,           /* unembedding fused with logsumexp_V (Eq. 6, Eq. 8) */
+  CPMTP_STAGE_MIXTURE,       /* Eq. 9 */
+  CPMTP_STAGE_FINALIZE,      /* loss, wbar, counts */
+  CPMTP_STAGE_COEFF,         /* backward coefficients */
+  CPMTP_STAGE_LOGIT_GRAD,    /* logits recompute -> dloss/dS */
+  CPMTP_STAGE_DZ,
+  CPMTP_STAGE_DE,
+  CPMTP_STAGE_DE_CONVERT,
+  CPMTP_STAGE_DW_HEAD,
+  CPMTP_STAGE_DH,
+  CPMTP_STAGE_DW_G,
+  CPMTP_STAGE_COUNT
+};
+int cpmtp_profile_begin(void);
+int cpmtp_profile_end(float* stage_ms, int32_t* stage_launches, int count);
+
 #ifdef __cplusplus
 }
 #endif

@@ -20,8 +20,12 @@ FLAG_AUX = 1
 
 EXPORTS = [
     "cpmtp_version", "cpmtp_status_string", "cpmtp_workspace_bytes", "cpmtp_forward", "cpmtp_backward",
-    "cpmtp_score_draft", "cpmtp_host_staging_bytes", "cpmtp_forward_host",
+    "cpmtp_score_draft", "cpmtp_host_staging_bytes", "cpmtp_forward_host", "cpmtp_profile_begin",
+    "cpmtp_profile_end",
 ]
+
+STAGES = ["gate", "proj", "lse", "mixture", "finalize", "coeff", "logit_grad", "dz", "de", "de_convert",
+          "dw_head", "dh", "dw_g"]
 
 
 class CShape(ctypes.Structure):
@@ -63,8 +67,26 @@ def load_library() -> ctypes.CDLL:
     lib.cpmtp_score_draft.argtypes = [shp, vp, vp, vp, vp, i32p, fp, fp, vp, sz, i32p, vp]
     lib.cpmtp_forward_host.restype = ctypes.c_int
     lib.cpmtp_forward_host.argtypes = [shp, vp, vp, vp, vp, i32p, fp, fp, svp, vp, sz, i32p, vp]
+    lib.cpmtp_profile_begin.restype = ctypes.c_int
+    lib.cpmtp_profile_end.restype = ctypes.c_int
+    lib.cpmtp_profile_end.argtypes = [ctypes.POINTER(ctypes.c_float), ctypes.POINTER(ctypes.c_int32), ctypes.c_int]
     _lib = lib
     return lib
+
+
+def profile_begin() -> None:
+    _check(load_library().cpmtp_profile_begin())
+
+
+def profile_end() -> dict:
+    """Stop per-stage timing; returns {stage: (total_ms, launches)} for stages that ran."""
+    n = len(STAGES)
+    ms = (ctypes.c_float * n)()
+    cnt = (ctypes.c_int32 * n)()
+    total = load_library().cpmtp_profile_end(ms, cnt, n)
+    if total < 0:
+        _check(total)
+    return {STAGES[i]: (float(ms[i]), int(cnt[i])) for i in range(n) if cnt[i] > 0}
 
 
 class CpmtpError(RuntimeError):
@@ -205,7 +227,7 @@ def score_draft(h, W_head, E, W_g, draft, *, want_prefix: bool = True,
 
 
 def forward_host(h_host, W_head, E, W_g, x_host, logp_host, loss_host, *, aux_coef: Optional[float] = None,
-                 workspace: Optional[torch.Tensor] = None, dev_status: Optional[torch.Tensor] = None) -> None:
+                 saved: Optional[Saved] = None, workspace: Optional[torch.Tensor] = None, dev_status: Optional[torch.Tensor] = None) -> None:
     """cpmtp_forward_host: h_host / x_host / logp_host / loss_host are (pinned) CPU tensors; weights on device.
     Asynchronous: synchronise the current stream before reading the host outputs."""
     lib = load_library()
@@ -214,7 +236,9 @@ def forward_host(h_host, W_head, E, W_g, x_host, logp_host, loss_host, *, aux_co
     need = workspace_bytes(shape, OP_FORWARD) + host_staging_bytes(shape) + 256
     if workspace is None:
         workspace = alloc_workspace(need, E.device)
+    cs = saved.c_struct() if saved is not None else None
     rc = lib.cpmtp_forward_host(ctypes.byref(shape), _ptr(h_host), _ptr(W_head), _ptr(E), _ptr(W_g), _ptr(x_host),
-                                _ptr(logp_host), _ptr(loss_host), None, _ptr(workspace), workspace.numel(),
+                                _ptr(logp_host), _ptr(loss_host), ctypes.byref(cs) if cs is not None else None,
+                                _ptr(workspace), workspace.numel(),
                                 _ptr(dev_status), _stream())
     _check(rc)

@@ -6,6 +6,7 @@
 #include <cuda_runtime.h>
 #include <cstdint>
 #include <cstdlib>
+#include <vector>
 
 #include "epilogues.cuh"
 #include "small_kernels.cuh"
@@ -137,6 +138,31 @@ BwdLayout bwd_layout(const cpmtp_shape& s) {
   return L;
 }
 
+// Optional per-stage timing: events bracket each launch while profiling is on.
+struct Profiler {
+  bool on = false;
+  std::vector<cudaEvent_t> events;   // start/stop pairs
+  std::vector<int> stages;
+};
+Profiler g_prof;
+
+struct ProfScope {
+  cudaStream_t st;
+  bool active;
+  ProfScope(int stage, cudaStream_t stream) : st(stream), active(g_prof.on) {
+    if (!active) return;
+    cudaEvent_t a, b;
+    if (cudaEventCreate(&a) != cudaSuccess || cudaEventCreate(&b) != cudaSuccess) { active = false; return; }
+    g_prof.events.push_back(a);
+    g_prof.events.push_back(b);
+    g_prof.stages.push_back(stage);
+    cudaEventRecord(a, st);
+  }
+  ~ProfScope() {
+    if (active) cudaEventRecord(g_prof.events.back(), st);
+  }
+};
+
 template <class Cfg, class Epi>
 cudaError_t launch_gemm(const void* A, uint64_t a_rows, uint64_t a_ld, const void* B, uint64_t b_rows,
                         uint64_t b_ld, uint64_t kdim, const Sched& sched, const typename Epi::Params& ep,
@@ -182,12 +208,14 @@ int run_forward(const cpmtp_shape& s, const uint16_t* h, const uint16_t* W_head,
 
   // gate (Eq. 7)
   {
+    ProfScope prof(CPMTP_STAGE_GATE, stream);
     const int warps = 8;
     gate_kernel<<<(s.N + warps - 1) / warps, warps * 32, 0, stream>>>(h, W_g, logw, s.N, s.d, s.r);
     CPMTP_TRY(cudaGetLastError());
   }
   // head projection: z[N, K*d] = h[N, d] * W_cat[K*d, d]^T, plus the fp32 target-logit partials
   {
+    ProfScope prof(CPMTP_STAGE_PROJ, stream);
     EpiProj<kBN>::Params ep{z, tgt_part, E, x, dev_status, s.N, ncols, s.d, s.V, s.n, s.r};
     const int m_tiles = (s.N + kBM - 1) / kBM;
     const int n_tiles = (ncols + kBN - 1) / kBN;
@@ -196,17 +224,20 @@ int run_forward(const cpmtp_shape& s, const uint16_t* h, const uint16_t* W_head,
   }
   // unembedding fused with the vocabulary log-sum-exp (Eq. 6, Eq. 8)
   {
+    ProfScope prof(CPMTP_STAGE_LSE, stream);
     EpiLse<kBN>::Params ep{part_m, part_l, L.M, s.V, L.lse_sched.n_splits};
     CPMTP_TRY((launch_gemm<CfgKK, EpiLse<kBN>>(z, L.M, s.d, E, s.V, s.d, s.d, L.lse_sched, ep, dev_status, sms, stream)));
   }
   // mixture epilogue (Eq. 9)
   {
+    ProfScope prof(CPMTP_STAGE_MIXTURE, stream);
     const int warps = 8;
     mixture_kernel<<<(s.N + warps - 1) / warps, warps * 32, 0, stream>>>(
         part_m, part_l, L.lse_sched.n_splits, tgt_part, s.d / 64, logw, lse, tgt, q, logp, logp_prefix, s.N, s.n, s.r);
     CPMTP_TRY(cudaGetLastError());
   }
   if (loss != nullptr || counts != nullptr || saved != nullptr) {
+    ProfScope prof(CPMTP_STAGE_FINALIZE, stream);
     const float aux = (s.flags & CPMTP_FLAG_AUX) ? s.aux_coef : 0.f;
     finalize_kernel<<<1, 1024, 0, stream>>>(logp, logw, wbar, counts, loss, s.N, s.r, aux);
     CPMTP_TRY(cudaGetLastError());
@@ -250,6 +281,38 @@ static int sms_or_default() {
 extern "C" {
 
 int cpmtp_version(void) { return 100; }
+
+int cpmtp_profile_begin(void) {
+  for (cudaEvent_t e : g_prof.events) cudaEventDestroy(e);
+  g_prof.events.clear();
+  g_prof.stages.clear();
+  g_prof.on = true;
+  return CPMTP_OK;
+}
+
+int cpmtp_profile_end(float* stage_ms, int32_t* stage_launches, int count) {
+  g_prof.on = false;
+  if (count < 0 || count > CPMTP_STAGE_COUNT) return CPMTP_ERR_SHAPE;
+  if (cudaDeviceSynchronize() != cudaSuccess) return CPMTP_ERR_LAUNCH;
+  for (int i = 0; i < count; ++i) {
+    if (stage_ms) stage_ms[i] = 0.f;
+    if (stage_launches) stage_launches[i] = 0;
+  }
+  const int total = static_cast<int>(g_prof.stages.size());
+  for (int j = 0; j < total; ++j) {
+    float ms = 0.f;
+    cudaEventElapsedTime(&ms, g_prof.events[2 * j], g_prof.events[2 * j + 1]);
+    const int stg = g_prof.stages[j];
+    if (stg < count) {
+      if (stage_ms) stage_ms[stg] += ms;
+      if (stage_launches) stage_launches[stg] += 1;
+    }
+  }
+  for (cudaEvent_t e : g_prof.events) cudaEventDestroy(e);
+  g_prof.events.clear();
+  g_prof.stages.clear();
+  return total;
+}
 
 const char* cpmtp_status_string(int status) {
   switch (status) {
@@ -373,9 +436,12 @@ int cpmtp_backward(const cpmtp_shape* shape, const void* h, const void* W_head, 
   const int ncols = K * d;
   const float aux = (s.flags & CPMTP_FLAG_AUX) ? s.aux_coef : 0.f;
 
-  coeff_kernel<<<(s.N + 255) / 256, 256, 0, st>>>(saved->q, saved->logw, saved->wbar, dloss_dlogp, coef, dg, s.N,
-                                                 s.r, aux);
-  CPMTP_TRY(cudaGetLastError());
+  {
+    ProfScope prof(CPMTP_STAGE_COEFF, st);
+    coeff_kernel<<<(s.N + 255) / 256, 256, 0, st>>>(saved->q, saved->logw, saved->wbar, dloss_dlogp, coef, dg,
+                                                   s.N, s.r, aux);
+    CPMTP_TRY(cudaGetLastError());
+  }
 
   const int d_tiles = (d + kBN - 1) / kBN;
   for (int c = 0; c < L.chunks; ++c) {
@@ -385,6 +451,7 @@ int cpmtp_backward(const cpmtp_shape* shape, const void* h, const void* W_head, 
     const int m_tiles = (rows + kBM - 1) / kBM;
     // recompute logits tile by tile -> G = dloss/dS (bf16), never more than one chunk
     {
+      ProfScope prof(CPMTP_STAGE_LOGIT_GRAD, st);
       EpiLogitGrad<kBN>::Params ep{G, saved->lse, coef, x, row0, rows, L.ldg, V, K, s.n, s.r};
       const int n_tiles = (L.ldg + kBN - 1) / kBN;
       const Sched sc = make_sched(m_tiles, n_tiles, n_tiles, 16, d / kBK);
@@ -392,12 +459,14 @@ int cpmtp_backward(const cpmtp_shape* shape, const void* h, const void* W_head, 
     }
     // dz[rows, d] = G[rows, V] * E[V, d]
     {
+      ProfScope prof(CPMTP_STAGE_DZ, st);
       EpiStoreBf16<kBN, false>::Params ep{dz + row0 * d, nullptr, nullptr, rows, d, d, 0};
       const Sched sc = make_sched(m_tiles, d_tiles, d_tiles, 16, (V + kBK - 1) / kBK);
       CPMTP_TRY((launch_gemm<CfgKM, EpiStoreBf16<kBN, false>>(G, rows, L.ldg, Eb, d, d, V, sc, ep, dev_status, sms, st)));
     }
     // dE[V, d] (+)= G^T[V, rows] * z[rows, d]
     {
+      ProfScope prof(CPMTP_STAGE_DE, st);
       const int v_tiles = (V + kBM - 1) / kBM;
       const Sched sc = make_sched(v_tiles, d_tiles, d_tiles, 16, (rows + kBK - 1) / kBK);
       if (L.chunks == 1) {
@@ -410,11 +479,13 @@ int cpmtp_backward(const cpmtp_shape* shape, const void* h, const void* W_head, 
     }
   }
   if (L.chunks > 1) {
+    ProfScope prof(CPMTP_STAGE_DE_CONVERT, st);
     f32_to_bf16_kernel<<<sms * 8, 256, 0, st>>>(dE32, static_cast<uint16_t*>(dE), static_cast<size_t>(V) * d);
     CPMTP_TRY(cudaGetLastError());
   }
   // dW_head[K*d, d] = dz^T[K*d, N] * h[N, d]
   {
+    ProfScope prof(CPMTP_STAGE_DW_HEAD, st);
     EpiStoreBf16<kBN, false>::Params ep{static_cast<uint16_t*>(dW_head), nullptr, nullptr, ncols, d, d, 0};
     const int m_tiles = (ncols + kBM - 1) / kBM;
     const Sched sc = make_sched(m_tiles, d_tiles, d_tiles, 16, (s.N + kBK - 1) / kBK);
@@ -422,6 +493,7 @@ int cpmtp_backward(const cpmtp_shape* shape, const void* h, const void* W_head, 
   }
   // dh[N, d] = dz[N, K*d] * W_cat[K*d, d] + dg * W_g
   {
+    ProfScope prof(CPMTP_STAGE_DH, st);
     EpiStoreBf16<kBN, true>::Params ep{static_cast<uint16_t*>(dh), dg, static_cast<const uint16_t*>(W_g), s.N, d, d, s.r};
     const int m_tiles = (s.N + kBM - 1) / kBM;
     const Sched sc = make_sched(m_tiles, d_tiles, d_tiles, 16, ncols / kBK);
@@ -429,6 +501,7 @@ int cpmtp_backward(const cpmtp_shape* shape, const void* h, const void* W_head, 
   }
   // dW_g[r, d] = dg^T * h
   {
+    ProfScope prof(CPMTP_STAGE_DW_G, st);
     dim3 grid((d + 127) / 128, L.dwg_slices);
     dwg_partial_kernel<CPMTP_MAX_R><<<grid, 128, 0, st>>>(dg, static_cast<const uint16_t*>(h), dwg_part, s.N, d, s.r,
                                                           L.dwg_rows_per_slice);

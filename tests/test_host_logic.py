@@ -1,0 +1,70 @@
+"""CPU-only checks: the C-ABI library loads, exports every declared symbol, sizes
+workspaces and rejects bad arguments before touching a GPU."""
+import ctypes
+import os
+import re
+
+import pytest
+
+from paper_2410_17765_b200 import binding, build
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+@pytest.fixture(scope="module")
+def lib():
+    build.build()
+    return binding.load_library()
+
+
+def test_exports_every_declared_symbol(lib):
+    header = open(os.path.join(ROOT, "include", "cpmtp.h")).read()
+    declared = set(re.findall(r"\b(cpmtp_[a-z_]+)\s*\(", header))
+    assert declared, "no declarations found"
+    assert declared == set(binding.EXPORTS)
+    for name in declared:
+        assert getattr(lib, name) is not None
+
+
+def test_version_and_status_strings(lib):
+    assert lib.cpmtp_version() >= 100
+    assert lib.cpmtp_status_string(0) == b"ok"
+    for code in range(-7, 0):
+        assert lib.cpmtp_status_string(code) not in (b"ok", b"unknown status")
+
+
+def test_workspace_sizes(lib):
+    s = binding.make_shape(64, 256, 1024, 3, 4)
+    fwd = binding.workspace_bytes(s, binding.OP_FORWARD)
+    bwd = binding.workspace_bytes(s, binding.OP_BACKWARD)
+    # forward holds at least z (bf16) ; backward at least dz and one 128-row chunk of logit gradients
+    assert fwd >= 2 * 64 * 12 * 256
+    assert bwd >= 2 * 64 * 12 * 256 + 2 * 128 * 1024
+    assert binding.workspace_bytes(s, binding.OP_SCORE) > 0
+    assert binding.workspace_bytes(s, 99) == 0
+    assert binding.host_staging_bytes(s) >= 2 * 64 * 256 + 4 * 64 * 3 + 4 * 64
+
+
+@pytest.mark.parametrize("bad", [dict(N=0), dict(d=100), dict(d=32), dict(V=1), dict(n=0), dict(n=9), dict(r=0), dict(r=33)])
+def test_invalid_shapes_are_rejected(lib, bad):
+    args = dict(N=8, d=128, V=100, n=2, r=2)
+    args.update(bad)
+    s = binding.make_shape(**args)
+    assert binding.workspace_bytes(s, binding.OP_FORWARD) == 0
+    buf = (ctypes.c_char * 4096)()
+    p = ctypes.cast(buf, ctypes.c_void_p)
+    rc = lib.cpmtp_forward(ctypes.byref(s), p, p, p, p, p, p, None, None, None, p, 4096, None, None)
+    assert rc == -2
+
+
+def test_null_and_misaligned_pointers_are_rejected(lib):
+    s = binding.make_shape(8, 128, 100, 2, 2)
+    buf = (ctypes.c_char * 8192)()
+    base = ctypes.addressof(buf)
+    base += (-base) % 256
+    p = ctypes.c_void_p(base)
+    odd = ctypes.c_void_p(base + 2)
+    assert lib.cpmtp_forward(ctypes.byref(s), None, p, p, p, p, p, None, None, None, p, 4096, None, None) == -1
+    assert lib.cpmtp_forward(ctypes.byref(s), odd, p, p, p, p, p, None, None, None, p, 4096, None, None) == -3
+    assert lib.cpmtp_backward(ctypes.byref(s), p, p, p, p, p, None, None, p, p, p, p, p, 4096, None, None) in (-1, -5, -6)
+    assert lib.cpmtp_forward(None, p, p, p, p, p, p, None, None, None, p, 4096, None, None) == -1
