@@ -62,18 +62,34 @@ inline bool aligned(const void* p, size_t a) { return (reinterpret_cast<uintptr_
 
 // Column-split schedule of the fused unembedding: `group` row tiles x `splits`
 // vocabulary ranges run concurrently, so the rows' z tiles stay L2-resident while
-// each range of E is streamed once per group.
-Sched sched_lse(int m_tiles, int n_tiles, int k_blocks, int sms) {
-  int splits, group;
-  if (m_tiles >= sms) {
-    splits = n_tiles < 4 ? n_tiles : 4;
-    group = sms / splits;
-  } else {
-    splits = (sms + m_tiles - 1) / m_tiles;
-    if (splits > n_tiles) splits = n_tiles;
-    group = m_tiles;
+// each range of E is streamed once per group.  The split count minimises a simple
+// time model: max(makespan of the tensor work, HBM traffic / bandwidth); ties go
+// to the choice that keeps more SMs busy, then to fewer splits.
+Sched sched_lse(int m_tiles, int n_tiles, int M, int V, int d, int sms) {
+  // keep the concurrently swept z tiles (group * 128 rows * d * 2 B) within ~64 MB of L2
+  int max_group = static_cast<int>((64ll << 20) / (256ll * d));
+  if (max_group < 1) max_group = 1;
+  const double tile_t = 2.0 * kBM * kBN * d / (1.4e15 / sms);
+  int best_s = 1, best_ctas = 0;
+  double best_score = -1.0;
+  const int s_max = n_tiles < sms ? n_tiles : sms;
+  for (int s = 1; s <= s_max; ++s) {
+    const int group = static_cast<long long>(m_tiles) * s >= sms ? (sms / s) : m_tiles;
+    if (group < 1 || group > max_group) continue;
+    const long long units = static_cast<long long>(m_tiles) * s;
+    const double comp = static_cast<double>((units + sms - 1) / sms) * ((n_tiles + s - 1) / s) * tile_t;
+    const double sweeps = (m_tiles + group - 1) / group;
+    const double mem = (sweeps * V * d * 2.0 + static_cast<double>(M) * d * 2.0) / 6.0e12;
+    const double score = (comp > mem ? comp : mem) + 0.1 * mem;
+    const int ctas = units < sms ? static_cast<int>(units) : sms;
+    if (best_score < 0 || score < best_score * 0.999 || (score <= best_score * 1.001 && ctas > best_ctas)) {
+      best_score = score;
+      best_s = s;
+      best_ctas = ctas;
+    }
   }
-  return make_sched(m_tiles, n_tiles, splits, group, k_blocks);
+  const int group = static_cast<long long>(m_tiles) * best_s >= sms ? (sms / best_s) : m_tiles;
+  return make_sched(m_tiles, n_tiles, best_s, group < 1 ? 1 : group, d / kBK);
 }
 
 struct FwdLayout {
@@ -88,7 +104,7 @@ FwdLayout fwd_layout(const cpmtp_shape& s, int sms) {
   L.M = s.N * L.K;
   const int m_tiles = (L.M + kBM - 1) / kBM;
   const int n_tiles = (s.V + kBN - 1) / kBN;
-  L.lse_sched = sched_lse(m_tiles, n_tiles, s.d / kBK, sms);
+  L.lse_sched = sched_lse(m_tiles, n_tiles, L.M, s.V, s.d, sms);
   size_t off = 0;
   auto take = [&](size_t bytes) { size_t o = off; off = align_up(off + bytes); return o; };
   L.logw = take(sizeof(float) * s.N * s.r);
@@ -209,8 +225,7 @@ int run_forward(const cpmtp_shape& s, const uint16_t* h, const uint16_t* W_head,
   // gate (Eq. 7)
   {
     ProfScope prof(CPMTP_STAGE_GATE, stream);
-    const int warps = 8;
-    gate_kernel<<<(s.N + warps - 1) / warps, warps * 32, 0, stream>>>(h, W_g, logw, s.N, s.d, s.r);
+    gate_kernel<<<s.N, 32 * s.r, 0, stream>>>(h, W_g, logw, s.N, s.d, s.r);
     CPMTP_TRY(cudaGetLastError());
   }
   // head projection: z[N, K*d] = h[N, d] * W_cat[K*d, d]^T, plus the fp32 target-logit partials
@@ -231,8 +246,7 @@ int run_forward(const cpmtp_shape& s, const uint16_t* h, const uint16_t* W_head,
   // mixture epilogue (Eq. 9)
   {
     ProfScope prof(CPMTP_STAGE_MIXTURE, stream);
-    const int warps = 8;
-    mixture_kernel<<<(s.N + warps - 1) / warps, warps * 32, 0, stream>>>(
+    mixture_kernel<<<s.N, 256, 0, stream>>>(
         part_m, part_l, L.lse_sched.n_splits, tgt_part, s.d / 64, logw, lse, tgt, q, logp, logp_prefix, s.N, s.n, s.r);
     CPMTP_TRY(cudaGetLastError());
   }

@@ -5,6 +5,7 @@
 #pragma once
 #include <cstdint>
 
+#include "../../include/cpmtp.h"
 #include "ptx.cuh"
 
 namespace cpmtp {
@@ -20,42 +21,44 @@ __device__ __forceinline__ float warp_max(float v) {
   return v;
 }
 
-// Gate of Eq. 7: logw[i, :] = log softmax(W_g h[i]).  One warp per position,
-// lane a ends up holding expert a (r <= 32).
+// Gate of Eq. 7: logw[i, :] = log softmax(W_g h[i]).  One block per position,
+// one warp per expert (blockDim.x = 32 * r, r <= 32).
 __global__ void gate_kernel(const uint16_t* __restrict__ h, const uint16_t* __restrict__ W_g,
                             float* __restrict__ logw, int N, int d, int r) {
-  const int warps_per_block = blockDim.x >> 5;
-  const int i = blockIdx.x * warps_per_block + (threadIdx.x >> 5);
+  __shared__ float g_s[32];
+  const int i = blockIdx.x;
+  const int a = threadIdx.x >> 5;
   const int lane = threadIdx.x & 31;
-  if (i >= N) return;
   const uint4* hrow = reinterpret_cast<const uint4*>(h + static_cast<size_t>(i) * d);
+  const uint4* wrow = reinterpret_cast<const uint4*>(W_g + static_cast<size_t>(a) * d);
   const int vecs = d >> 3;
-  float mine = -INFINITY;
-  for (int a = 0; a < r; ++a) {
-    const uint4* wrow = reinterpret_cast<const uint4*>(W_g + static_cast<size_t>(a) * d);
-    float acc = 0.f;
-    for (int j = lane; j < vecs; j += 32) {
-      const uint4 hv = __ldg(hrow + j);
-      const uint4 wv = __ldg(wrow + j);
-      acc = fmaf(ptx::bf16_lo(hv.x), ptx::bf16_lo(wv.x), acc);
-      acc = fmaf(ptx::bf16_hi(hv.x), ptx::bf16_hi(wv.x), acc);
-      acc = fmaf(ptx::bf16_lo(hv.y), ptx::bf16_lo(wv.y), acc);
-      acc = fmaf(ptx::bf16_hi(hv.y), ptx::bf16_hi(wv.y), acc);
-      acc = fmaf(ptx::bf16_lo(hv.z), ptx::bf16_lo(wv.z), acc);
-      acc = fmaf(ptx::bf16_hi(hv.z), ptx::bf16_hi(wv.z), acc);
-      acc = fmaf(ptx::bf16_lo(hv.w), ptx::bf16_lo(wv.w), acc);
-      acc = fmaf(ptx::bf16_hi(hv.w), ptx::bf16_hi(wv.w), acc);
-    }
-    acc = warp_sum(acc);
-    if (lane == a) mine = acc;
+  float acc = 0.f;
+  for (int j = lane; j < vecs; j += 32) {
+    const uint4 hv = __ldg(hrow + j);
+    const uint4 wv = __ldg(wrow + j);
+    acc = fmaf(ptx::bf16_lo(hv.x), ptx::bf16_lo(wv.x), acc);
+    acc = fmaf(ptx::bf16_hi(hv.x), ptx::bf16_hi(wv.x), acc);
+    acc = fmaf(ptx::bf16_lo(hv.y), ptx::bf16_lo(wv.y), acc);
+    acc = fmaf(ptx::bf16_hi(hv.y), ptx::bf16_hi(wv.y), acc);
+    acc = fmaf(ptx::bf16_lo(hv.z), ptx::bf16_lo(wv.z), acc);
+    acc = fmaf(ptx::bf16_hi(hv.z), ptx::bf16_hi(wv.z), acc);
+    acc = fmaf(ptx::bf16_lo(hv.w), ptx::bf16_lo(wv.w), acc);
+    acc = fmaf(ptx::bf16_hi(hv.w), ptx::bf16_hi(wv.w), acc);
   }
-  const float m = warp_max(mine);
-  const float e = lane < r ? expf(mine - m) : 0.f;
-  const float lse = m + logf(warp_sum(e));
-  if (lane < r) logw[static_cast<size_t>(i) * r + lane] = mine - lse;
+  acc = warp_sum(acc);
+  if (lane == 0) g_s[a] = acc;
+  __syncthreads();
+  if (a == 0) {
+    const float mine = lane < r ? g_s[lane] : -INFINITY;
+    const float m = warp_max(mine);
+    const float e = lane < r ? expf(mine - m) : 0.f;
+    const float lse = m + logf(warp_sum(e));
+    if (lane < r) logw[static_cast<size_t>(i) * r + lane] = mine - lse;
+  }
 }
 
-// Mixture epilogue (last line of Eq. 9).  One warp per position.
+// Mixture epilogue (last line of Eq. 9).  One block per position; warps share the
+// n*r heads, then warp 0 mixes the experts (lane = expert).
 //   lse[i,k]  = two-pass merge of the per-split (max, sum-exp) partials
 //   tgt[i,k]  = sum of the per-64-column target-logit partials
 //   a[i,al]   = logw[i,al] + sum_s (tgt - lse)[i, s*r+al]
@@ -67,34 +70,37 @@ __global__ void mixture_kernel(const float* __restrict__ part_m, const float* __
                                float* __restrict__ tgt_out, float* __restrict__ q_out,
                                float* __restrict__ logp, float* __restrict__ logp_prefix, int N, int n,
                                int r) {
-  const int warps_per_block = blockDim.x >> 5;
-  const int i = blockIdx.x * warps_per_block + (threadIdx.x >> 5);
+  __shared__ float c_s[CPMTP_MAX_N * CPMTP_MAX_R];
+  const int i = blockIdx.x;
+  const int warp = threadIdx.x >> 5;
+  const int nwarps = blockDim.x >> 5;
   const int lane = threadIdx.x & 31;
-  if (i >= N) return;
   const int K = n * r;
+  for (int k = warp; k < K; k += nwarps) {
+    const size_t row = static_cast<size_t>(i) * K + k;
+    // pass 1: global max over splits; pass 2: rescaled sum
+    float m = -INFINITY;
+    for (int j = lane; j < splits; j += 32) m = fmaxf(m, part_m[row * splits + j]);
+    m = warp_max(m);
+    float l = 0.f;
+    for (int j = lane; j < splits; j += 32)
+      l += part_l[row * splits + j] * exp2f(part_m[row * splits + j] - m);
+    l = warp_sum(l);
+    const float lse = (m + log2f(l)) * 0.6931471805599453f;
+    float t = 0.f;
+    for (int j = lane; j < tgt_parts; j += 32) t += tgt_part[row * tgt_parts + j];
+    t = warp_sum(t);
+    if (lane == 0) {
+      c_s[k] = t - lse;
+      if (lse_out != nullptr) lse_out[row] = lse;
+      if (tgt_out != nullptr) tgt_out[row] = t;
+    }
+  }
+  __syncthreads();
+  if (warp != 0) return;
   float a = lane < r ? logw[static_cast<size_t>(i) * r + lane] : -INFINITY;
   for (int s = 0; s < n; ++s) {
-    for (int al = 0; al < r; ++al) {
-      const int k = s * r + al;
-      const size_t row = static_cast<size_t>(i) * K + k;
-      // pass 1: global max over splits; pass 2: rescaled sum
-      float m = -INFINITY;
-      for (int j = lane; j < splits; j += 32) m = fmaxf(m, part_m[row * splits + j]);
-      m = warp_max(m);
-      float l = 0.f;
-      for (int j = lane; j < splits; j += 32)
-        l += part_l[row * splits + j] * exp2f(part_m[row * splits + j] - m);
-      l = warp_sum(l);
-      const float lse = (m + log2f(l)) * 0.6931471805599453f;
-      float t = 0.f;
-      for (int j = lane; j < tgt_parts; j += 32) t += tgt_part[row * tgt_parts + j];
-      t = warp_sum(t);
-      if (lane == al) {
-        a += t - lse;
-        if (lse_out != nullptr) lse_out[row] = lse;
-        if (tgt_out != nullptr) tgt_out[row] = t;
-      }
-    }
+    if (lane < r) a += c_s[s * r + lane];
     if (logp_prefix != nullptr || s == n - 1) {
       const float m = warp_max(a);
       const float e = lane < r ? expf(a - m) : 0.f;
