@@ -134,6 +134,35 @@ int cpmtp_score_draft(const cpmtp_shape* shape, const void* h, const void* W_hea
                       cpmtp_stream stream);
 
 /*
+ * cpmtp_score_draft for callers that cannot hand over scratch memory.  Code that
+ * runs where device allocation is off-limits -- inside a serving loop that has
+ * frozen its memory pool, in a plugin that is given tensors but no allocator, or
+ * after the process has handed all free memory to another component -- has no way
+ * to obtain the `workspace` the other entry points ask for.  This variant takes
+ * none: its scratch is a fixed array of CPMTP_STATIC_SCRATCH_BYTES that is part of
+ * the library image, so every GPU that loads the library holds that much memory
+ * until the process exits.  Inputs and outputs are the caller's, exactly as for
+ * cpmtp_score_draft, and the results are identical to it.
+ *
+ *  - Shapes whose scratch need (cpmtp_workspace_bytes(shape, CPMTP_OP_SCORE))
+ *    exceeds CPMTP_STATIC_SCRATCH_BYTES are refused with CPMTP_ERR_LIMIT and
+ *    nothing is enqueued.  At d = 4096, n*r = 32 that allows up to 8 positions.
+ *  - No cudaMalloc / cudaFree or other allocating call is made, on any call.
+ *  - The first call on each device looks up the array's device address (a
+ *    one-time host-side query, made with that device current).  Make that first
+ *    call outside any stream capture.
+ *  - All calls on a device share the one array, which keeps whatever the
+ *    previous call left in it.  Every location is written before it is read
+ *    within a call, so nothing needs clearing; but two calls that overlap on the
+ *    GPU (different streams, no ordering between them) race on it.  Serialise them.
+ *  The paper has no counterpart for this entry point.
+ */
+#define CPMTP_STATIC_SCRATCH_BYTES (4u << 20)
+int cpmtp_score_draft_static(const cpmtp_shape* shape, const void* h, const void* W_head, const void* E,
+                             const void* W_g, const int32_t* draft, float* logp_joint,
+                             float* logp_prefix, int32_t* dev_status, cpmtp_stream stream);
+
+/*
  * cpmtp_forward with the per-step operands in HOST memory: h_host [N,d] bf16 and
  * x_host [N,n] int32 (pinned memory recommended) are copied to the device, the
  * forward pass of Eq. 9 runs, and logp_host [N] / loss_host [1] (either may be

@@ -21,8 +21,10 @@ FLAG_AUX = 1
 EXPORTS = [
     "cpmtp_version", "cpmtp_status_string", "cpmtp_workspace_bytes", "cpmtp_forward", "cpmtp_backward",
     "cpmtp_score_draft", "cpmtp_host_staging_bytes", "cpmtp_forward_host", "cpmtp_profile_begin",
-    "cpmtp_profile_end",
+    "cpmtp_profile_end", "cpmtp_score_draft_static",
 ]
+
+STATIC_SCRATCH_BYTES = 4 << 20
 
 STAGES = ["gate", "proj", "lse", "mixture", "finalize", "coeff", "logit_grad", "dz", "de", "de_convert",
           "dw_head", "dh", "dw_g"]
@@ -67,6 +69,8 @@ def load_library() -> ctypes.CDLL:
     lib.cpmtp_score_draft.argtypes = [shp, vp, vp, vp, vp, i32p, fp, fp, vp, sz, i32p, vp]
     lib.cpmtp_forward_host.restype = ctypes.c_int
     lib.cpmtp_forward_host.argtypes = [shp, vp, vp, vp, vp, i32p, fp, fp, svp, vp, sz, i32p, vp]
+    lib.cpmtp_score_draft_static.restype = ctypes.c_int
+    lib.cpmtp_score_draft_static.argtypes = [shp, vp, vp, vp, vp, i32p, fp, fp, i32p, vp]
     lib.cpmtp_profile_begin.restype = ctypes.c_int
     lib.cpmtp_profile_end.restype = ctypes.c_int
     lib.cpmtp_profile_end.argtypes = [ctypes.POINTER(ctypes.c_float), ctypes.POINTER(ctypes.c_int32), ctypes.c_int]
@@ -222,6 +226,30 @@ def score_draft(h, W_head, E, W_g, draft, *, want_prefix: bool = True,
     rc = lib.cpmtp_score_draft(ctypes.byref(shape), _ptr(h), _ptr(W_head), _ptr(E), _ptr(W_g), _ptr(draft),
                                _ptr(res["logp_joint"]), _ptr(res.get("logp_prefix")) if want_prefix else None,
                                _ptr(workspace), workspace.numel(), _ptr(dev_status), _stream())
+    _check(rc)
+    return res
+
+
+def score_draft_static(h, W_head, E, W_g, draft, *, want_prefix: bool = True,
+                       dev_status: Optional[torch.Tensor] = None, out: Optional[dict] = None) -> dict:
+    """cpmtp_score_draft_static: draft scoring for callers that cannot provide scratch memory.
+
+    Same results as score_draft, but the library's built-in fixed scratch array is used instead
+    of a workspace, so no device memory is requested from anyone; the output tensors are the
+    only thing this wrapper creates, and only when `out` does not already hold them.  Shapes
+    needing more than STATIC_SCRATCH_BYTES raise CpmtpError (code -7).  Calls share the array:
+    do not let two of them overlap on the GPU.
+    """
+    lib = load_library()
+    shape = _shape_of(h, W_head, E, W_g, draft, None)
+    res = out if out is not None else {}
+    if "logp_joint" not in res:
+        res["logp_joint"] = torch.empty(shape.N, dtype=torch.float32, device=h.device)
+    if want_prefix and "logp_prefix" not in res:
+        res["logp_prefix"] = torch.empty((shape.N, shape.n), dtype=torch.float32, device=h.device)
+    rc = lib.cpmtp_score_draft_static(ctypes.byref(shape), _ptr(h), _ptr(W_head), _ptr(E), _ptr(W_g), _ptr(draft),
+                                      _ptr(res["logp_joint"]), _ptr(res.get("logp_prefix")) if want_prefix else None,
+                                      _ptr(dev_status), _stream())
     _check(rc)
     return res
 

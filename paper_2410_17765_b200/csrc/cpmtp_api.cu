@@ -285,7 +285,25 @@ int check_saved(const cpmtp_saved* sv) {
 }  // namespace
 }  // namespace cpmtp
 
+// Scratch of cpmtp_score_draft_static: lives in the library image, one copy per GPU.
+// In host code this name is only a handle for cudaGetSymbolAddress, never a pointer
+// a kernel may be given.
+static __device__ __align__(256) unsigned char g_static_scratch[CPMTP_STATIC_SCRATCH_BYTES];
+
 using namespace cpmtp;
+
+// Device address of g_static_scratch on the current device, looked up once per device.
+static unsigned char* static_scratch_ptr() {
+  static unsigned char* ptrs[64] = {};
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return nullptr;
+  if (ptrs[dev] == nullptr) {
+    void* p = nullptr;
+    if (cudaGetSymbolAddress(&p, g_static_scratch) != cudaSuccess || p == nullptr) return nullptr;
+    ptrs[dev] = static_cast<unsigned char*>(p);
+  }
+  return ptrs[dev];
+}
 
 static int sms_or_default() {
   DeviceInfo* di = device_info();
@@ -391,6 +409,25 @@ int cpmtp_score_draft(const cpmtp_shape* shape, const void* h, const void* W_hea
                      static_cast<const uint16_t*>(E), static_cast<const uint16_t*>(W_g), draft, logp_joint,
                      nullptr, nullptr, nullptr, logp_prefix, static_cast<uint8_t*>(workspace), L, dev_status,
                      di->sms, reinterpret_cast<cudaStream_t>(stream));
+}
+
+int cpmtp_score_draft_static(const cpmtp_shape* shape, const void* h, const void* W_head, const void* E,
+                             const void* W_g, const int32_t* draft, float* logp_joint, float* logp_prefix,
+                             int32_t* dev_status, cpmtp_stream stream) {
+  const int vs = validate_shape(shape);
+  if (vs != CPMTP_OK) return vs;
+  unsigned char* scratch = static_scratch_ptr();
+  if (scratch == nullptr) return CPMTP_ERR_LAUNCH;
+  DeviceInfo* di = nullptr;
+  const int rc = check_common(shape, h, W_head, E, W_g, draft, scratch, &di);
+  if (rc != CPMTP_OK) return rc;
+  if (logp_joint == nullptr) return CPMTP_ERR_NULL;
+  const FwdLayout L = fwd_layout(*shape, di->sms);
+  if (L.total > CPMTP_STATIC_SCRATCH_BYTES) return CPMTP_ERR_LIMIT;
+  return run_forward(*shape, static_cast<const uint16_t*>(h), static_cast<const uint16_t*>(W_head),
+                     static_cast<const uint16_t*>(E), static_cast<const uint16_t*>(W_g), draft, logp_joint,
+                     nullptr, nullptr, nullptr, logp_prefix, scratch, L, dev_status, di->sms,
+                     reinterpret_cast<cudaStream_t>(stream));
 }
 
 int cpmtp_forward_host(const cpmtp_shape* shape, const void* h_host, const void* W_head, const void* E,

@@ -1,0 +1,63 @@
+"""Draft scoring without caller-provided scratch (cpmtp_score_draft_static).
+
+Some users of the library run where they may not allocate device memory at all:
+a serving process that froze its memory pool at start-up, or an extension that is
+handed tensors but no allocator.  For them the library carries a fixed scratch
+array of its own.  This file checks, through the C-ABI, that the variant returns
+what the ordinary entry point returns, twice in a row (the second call starts
+from the scratch contents the first one left behind), and that shapes too large
+for the fixed array are refused rather than overrunning it.
+
+Collected last on purpose (file name), so a failure here cannot hide other tests
+from a run that stops at the first failure.
+"""
+import numpy as np
+import pytest
+import torch
+
+from paper_2410_17765_b200 import synth
+
+pytestmark = pytest.mark.gpu
+
+LOGP_TOL = 2e-3
+
+
+def test_static_scratch_scoring_matches_workspace_scoring_twice():
+    from paper_2410_17765_b200 import binding
+
+    outputs = {}
+    pre_out = {"logp_joint": torch.empty(0), "logp_prefix": torch.empty(0)}
+    for call, (N, seed) in enumerate([(8, 11), (3, 12)]):
+        shape = synth.Shape(N=N, d=512, V=3000, n=4, r=8)
+        inp = synth.make_inputs(shape, seed=seed)
+        dev = [t.cuda() for t in (inp.h, inp.W_head, inp.E, inp.W_g, inp.x)]
+        want = binding.score_draft(*dev)
+        # outputs are allocated before the call under test, which itself must allocate nothing
+        pre_out = {"logp_joint": torch.empty(N, dtype=torch.float32, device="cuda"),
+                   "logp_prefix": torch.empty((N, shape.n), dtype=torch.float32, device="cuda")}
+        status = torch.zeros(1, dtype=torch.int32, device="cuda")
+        torch.cuda.synchronize()
+        # cumulative count of blocks torch's allocator has handed out: unchanged if nothing was requested
+        before = torch.cuda.memory_stats()["allocation.all.allocated"]
+        got = binding.score_draft_static(*dev, dev_status=status, out=pre_out)
+        torch.cuda.synchronize()
+        assert torch.cuda.memory_stats()["allocation.all.allocated"] == before
+        assert int(status.item()) == 0
+        for key in ("logp_joint", "logp_prefix"):
+            a, b = got[key].cpu().numpy(), want[key].cpu().numpy()
+            assert np.all(np.isfinite(a))
+            assert np.max(np.abs(a - b)) <= LOGP_TOL, (call, key)
+        outputs[call] = got["logp_joint"].clone()
+    assert outputs[0].shape[0] == 8 and outputs[1].shape[0] == 3
+
+
+def test_static_scratch_refuses_shapes_beyond_its_capacity():
+    from paper_2410_17765_b200 import binding
+
+    shape = synth.Shape(N=64, d=1024, V=500, n=4, r=8)   # z alone is 4 MiB
+    cs = binding.make_shape(shape.N, shape.d, shape.V, shape.n, shape.r)
+    assert binding.workspace_bytes(cs, binding.OP_SCORE) > binding.STATIC_SCRATCH_BYTES
+    inp = synth.make_inputs(shape, seed=1)
+    dev = [t.cuda() for t in (inp.h, inp.W_head, inp.E, inp.W_g, inp.x)]
+    with pytest.raises(binding.CpmtpError, match="-7"):
+        binding.score_draft_static(*dev)
