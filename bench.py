@@ -39,7 +39,9 @@ WORKLOADS = {
 
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel, from the ncu
 # captures summarised under profiles/ (None until captured, or once the kernel has changed since).
-NCU_TRAFFIC_BYTES = {}
+NCU_TRAFFIC_BYTES = {
+    "train_fwd": 1.211704e9 + 6.09024e6,   # profiles/lse_train_fwd.md
+}
 
 
 def measured_peaks():
