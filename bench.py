@@ -171,21 +171,17 @@ def run_reference(args, rank: int):
 def run_ours(args, rank: int, world: int, local_rank: int):
     import torch
 
-    from paper_2410_17765_b200 import binding, synth
+    from paper_2410_17765_b200 import binding, dist_util, synth
 
     if not torch.cuda.is_available():
         raise RuntimeError("bench.py needs a CUDA device; there is no CPU fallback")
     torch.cuda.set_device(local_rank)
-    dist = None
-    if world > 1:
-        import torch.distributed as dist_mod
-
-        dist = dist_mod
-        dist.init_process_group(backend="nccl", device_id=torch.device("cuda", local_rank))
+    device = torch.device("cuda", local_rank)
+    dist_util.init("nccl", device)
 
     cfg, kind, extra, aux = WORKLOADS[args.workload]
     shape = synth.CONFIGS[cfg]
-    inp = synth.make_inputs(shape, seed=rank, **extra)
+    inp = synth.make_inputs(shape, seed=dist_util.shard_seed(0, rank), **extra)
     h, W_head, E, W_g, x = [t.cuda() for t in (inp.h, inp.W_head, inp.E, inp.W_g, inp.x)]
     cs = binding.make_shape(shape.N, shape.d, shape.V, shape.n, shape.r, aux)
     ws_fwd = binding.alloc_workspace(binding.workspace_bytes(cs, binding.OP_FORWARD) +
@@ -220,9 +216,8 @@ def run_ours(args, rank: int, world: int, local_rank: int):
 
     def barrier():
         torch.cuda.synchronize()
-        if dist is not None:
-            dist.barrier()
-            torch.cuda.synchronize()
+        dist_util.barrier()
+        torch.cuda.synchronize()
 
     def timed(fn, steps, profile):
         barrier()
@@ -237,11 +232,7 @@ def run_ours(args, rank: int, world: int, local_rank: int):
         stages = binding.profile_end() if profile else {}
         ms = e0.elapsed_time(e1)
         barrier()
-        if dist is not None:
-            t = torch.tensor([ms], device="cuda", dtype=torch.float64)
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-            ms = float(t.item())
-        return ms, stages
+        return dist_util.max_over_ranks(ms, device), stages
 
     for _ in range(args.warmup):
         step()
@@ -255,13 +246,12 @@ def run_ours(args, rank: int, world: int, local_rank: int):
         raise RuntimeError(f"device status {int(status.item())} raised during the benchmark")
 
     if rank != 0:
-        if dist is not None:
-            dist.destroy_process_group()
+        dist_util.finalize()
         return
     peaks = measured_peaks()
     positions = shape.N * world
-    value = positions * args.steps / (ms_total * 1e-3)
-    e2e_value = positions * args.steps / (ms_e2e * 1e-3)
+    value = dist_util.whole_job_rate(shape.N, args.steps, world, ms_total)
+    e2e_value = dist_util.whole_job_rate(shape.N, args.steps, world, ms_e2e)
     K = shape.n * shape.r
     dominant = "lse"
     dom_ms, dom_launches = stages.get(dominant, (0.0, 0))
@@ -302,8 +292,7 @@ def run_ours(args, rank: int, world: int, local_rank: int):
         "stages_ms_per_step": {k: v[0] / args.steps for k, v in stages.items()},
     }
     print(json.dumps(line))
-    if dist is not None:
-        dist.destroy_process_group()
+    dist_util.finalize()
 
 
 def main():

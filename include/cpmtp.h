@@ -189,10 +189,10 @@ int cpmtp_forward_host(const cpmtp_shape* shape, const void* h_host, const void*
  * time.  The paper has no counterpart for these two calls.
  */
 enum {
-  CPMTP_STAGE_GATE = 0,      /* Eq. 7 */
+  CPMTP_STAGE_GATE = 0,      /* unused: the gate of Eq. 7 runs inside the mixture launch */
   CPMTP_STAGE_PROJ,          /* head projection + target-logit partials */
   CPMTP_STAGE_LSE,           /* unembedding fused with logsumexp_V (Eq. 6, Eq. 8) */
-  CPMTP_STAGE_MIXTURE,       /* Eq. 9 */
+  CPMTP_STAGE_MIXTURE,       /* Eq. 7 + Eq. 9 */
   CPMTP_STAGE_FINALIZE,      /* loss, wbar, counts */
   CPMTP_STAGE_COEFF,         /* backward coefficients */
   CPMTP_STAGE_LOGIT_GRAD,    /* logits recompute -> dloss/dS */

@@ -22,6 +22,7 @@ constexpr size_t kAlign = 256;
 constexpr size_t kLogitGradBudgetBytes = 4ull << 30;   // bound on the recomputed-logit-gradient chunk
 
 using CfgKK = TileCfg<kBN, kStages, false, false>;   // A K-major, B K-major
+using CfgKKSkinny = TileCfg<kBN, 5, false, false, 32>;   // <= 32 rows of A: bandwidth-bound draft scoring
 using CfgKM = TileCfg<kBN, kStages, false, true>;    // A K-major, B MN-major
 using CfgMM = TileCfg<kBN, kStages, true, true>;     // both MN-major
 
@@ -65,11 +66,11 @@ inline bool aligned(const void* p, size_t a) { return (reinterpret_cast<uintptr_
 // each range of E is streamed once per group.  The split count minimises a simple
 // time model: max(makespan of the tensor work, HBM traffic / bandwidth); ties go
 // to the choice that keeps more SMs busy, then to fewer splits.
-Sched sched_lse(int m_tiles, int n_tiles, int M, int V, int d, int sms) {
+Sched sched_lse(int m_tiles, int n_tiles, int M, int V, int d, int bn, int sms) {
   // keep the concurrently swept z tiles (group * 128 rows * d * 2 B) within ~64 MB of L2
   int max_group = static_cast<int>((64ll << 20) / (256ll * d));
   if (max_group < 1) max_group = 1;
-  const double tile_t = 2.0 * kBM * kBN * d / (1.4e15 / sms);
+  const double tile_t = 2.0 * kBM * bn * d / (1.4e15 / sms);
   int best_s = 1, best_ctas = 0;
   double best_score = -1.0;
   const int s_max = n_tiles < sms ? n_tiles : sms;
@@ -104,7 +105,7 @@ FwdLayout fwd_layout(const cpmtp_shape& s, int sms) {
   L.M = s.N * L.K;
   const int m_tiles = (L.M + kBM - 1) / kBM;
   const int n_tiles = (s.V + kBN - 1) / kBN;
-  L.lse_sched = sched_lse(m_tiles, n_tiles, L.M, s.V, s.d, sms);
+  L.lse_sched = sched_lse(m_tiles, n_tiles, L.M, s.V, s.d, kBN, sms);
   size_t off = 0;
   auto take = [&](size_t bytes) { size_t o = off; off = align_up(off + bytes); return o; };
   L.logw = take(sizeof(float) * s.N * s.r);
@@ -185,7 +186,7 @@ cudaError_t launch_gemm(const void* A, uint64_t a_rows, uint64_t a_ld, const voi
                         int* dev_status, int sms, cudaStream_t stream) {
   static bool attr_set[64] = {};
   CUtensorMap tA, tB;
-  if (!make_operand_tmap(&tA, A, Cfg::A_MN, a_rows, kdim, a_ld, kBM)) return cudaErrorInvalidValue;
+  if (!make_operand_tmap(&tA, A, Cfg::A_MN, a_rows, kdim, a_ld, Cfg::A_ROWS)) return cudaErrorInvalidValue;
   if (!make_operand_tmap(&tB, B, Cfg::B_MN, b_rows, kdim, b_ld, Cfg::BN)) return cudaErrorInvalidValue;
   constexpr int smem = gemm_smem_bytes<Cfg, Epi>();
   int dev = 0;
@@ -222,32 +223,35 @@ int run_forward(const cpmtp_shape& s, const uint16_t* h, const uint16_t* W_head,
   const int K = L.K;
   const int ncols = K * s.d;
 
-  // gate (Eq. 7)
-  {
-    ProfScope prof(CPMTP_STAGE_GATE, stream);
-    gate_kernel<<<s.N, 32 * s.r, 0, stream>>>(h, W_g, logw, s.N, s.d, s.r);
-    CPMTP_TRY(cudaGetLastError());
-  }
   // head projection: z[N, K*d] = h[N, d] * W_cat[K*d, d]^T, plus the fp32 target-logit partials
   {
     ProfScope prof(CPMTP_STAGE_PROJ, stream);
-    EpiProj<kBN>::Params ep{z, tgt_part, E, x, dev_status, s.N, ncols, s.d, s.V, s.n, s.r};
     const int m_tiles = (s.N + kBM - 1) / kBM;
     const int n_tiles = (ncols + kBN - 1) / kBN;
     const Sched sc = make_sched(m_tiles, n_tiles, n_tiles, m_tiles < 64 ? m_tiles : 64, s.d / kBK);
-    CPMTP_TRY((launch_gemm<CfgKK, EpiProj<kBN>>(h, s.N, s.d, W_head, ncols, s.d, s.d, sc, ep, dev_status, sms, stream)));
+    EpiProj<kBN>::Params ep{z, tgt_part, E, x, dev_status, s.N, ncols, s.d, s.V, s.n, s.r};
+    if (s.N <= CfgKKSkinny::A_ROWS) {
+      CPMTP_TRY((launch_gemm<CfgKKSkinny, EpiProj<kBN>>(h, s.N, s.d, W_head, ncols, s.d, s.d, sc, ep, dev_status, sms, stream)));
+    } else {
+      CPMTP_TRY((launch_gemm<CfgKK, EpiProj<kBN>>(h, s.N, s.d, W_head, ncols, s.d, s.d, sc, ep, dev_status, sms, stream)));
+    }
   }
   // unembedding fused with the vocabulary log-sum-exp (Eq. 6, Eq. 8)
   {
     ProfScope prof(CPMTP_STAGE_LSE, stream);
     EpiLse<kBN>::Params ep{part_m, part_l, L.M, s.V, L.lse_sched.n_splits};
-    CPMTP_TRY((launch_gemm<CfgKK, EpiLse<kBN>>(z, L.M, s.d, E, s.V, s.d, s.d, L.lse_sched, ep, dev_status, sms, stream)));
+    if (L.M <= CfgKKSkinny::A_ROWS) {
+      CPMTP_TRY((launch_gemm<CfgKKSkinny, EpiLse<kBN>>(z, L.M, s.d, E, s.V, s.d, s.d, L.lse_sched, ep, dev_status, sms, stream)));
+    } else {
+      CPMTP_TRY((launch_gemm<CfgKK, EpiLse<kBN>>(z, L.M, s.d, E, s.V, s.d, s.d, L.lse_sched, ep, dev_status, sms, stream)));
+    }
   }
-  // mixture epilogue (Eq. 9)
+  // gate (Eq. 7) and mixture epilogue (Eq. 9)
   {
     ProfScope prof(CPMTP_STAGE_MIXTURE, stream);
-    mixture_kernel<<<s.N, 256, 0, stream>>>(
-        part_m, part_l, L.lse_sched.n_splits, tgt_part, s.d / 64, logw, lse, tgt, q, logp, logp_prefix, s.N, s.n, s.r);
+    const int threads = s.N <= 256 ? 1024 : 256;
+    gate_mixture_kernel<<<s.N, threads, 0, stream>>>(h, W_g, s.d, part_m, part_l, L.lse_sched.n_splits, tgt_part,
+                                                    s.d / 64, logw, lse, tgt, q, logp, logp_prefix, s.N, s.n, s.r);
     CPMTP_TRY(cudaGetLastError());
   }
   if (loss != nullptr || counts != nullptr || saved != nullptr) {

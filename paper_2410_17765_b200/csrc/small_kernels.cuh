@@ -21,64 +21,55 @@ __device__ __forceinline__ float warp_max(float v) {
   return v;
 }
 
-// Gate of Eq. 7: logw[i, :] = log softmax(W_g h[i]).  One block per position,
-// one warp per expert (blockDim.x = 32 * r, r <= 32).
-__global__ void gate_kernel(const uint16_t* __restrict__ h, const uint16_t* __restrict__ W_g,
-                            float* __restrict__ logw, int N, int d, int r) {
-  __shared__ float g_s[32];
-  const int i = blockIdx.x;
-  const int a = threadIdx.x >> 5;
-  const int lane = threadIdx.x & 31;
-  const uint4* hrow = reinterpret_cast<const uint4*>(h + static_cast<size_t>(i) * d);
-  const uint4* wrow = reinterpret_cast<const uint4*>(W_g + static_cast<size_t>(a) * d);
-  const int vecs = d >> 3;
-  float acc = 0.f;
-  for (int j = lane; j < vecs; j += 32) {
-    const uint4 hv = __ldg(hrow + j);
-    const uint4 wv = __ldg(wrow + j);
-    acc = fmaf(ptx::bf16_lo(hv.x), ptx::bf16_lo(wv.x), acc);
-    acc = fmaf(ptx::bf16_hi(hv.x), ptx::bf16_hi(wv.x), acc);
-    acc = fmaf(ptx::bf16_lo(hv.y), ptx::bf16_lo(wv.y), acc);
-    acc = fmaf(ptx::bf16_hi(hv.y), ptx::bf16_hi(wv.y), acc);
-    acc = fmaf(ptx::bf16_lo(hv.z), ptx::bf16_lo(wv.z), acc);
-    acc = fmaf(ptx::bf16_hi(hv.z), ptx::bf16_hi(wv.z), acc);
-    acc = fmaf(ptx::bf16_lo(hv.w), ptx::bf16_lo(wv.w), acc);
-    acc = fmaf(ptx::bf16_hi(hv.w), ptx::bf16_hi(wv.w), acc);
-  }
-  acc = warp_sum(acc);
-  if (lane == 0) g_s[a] = acc;
-  __syncthreads();
-  if (a == 0) {
-    const float mine = lane < r ? g_s[lane] : -INFINITY;
-    const float m = warp_max(mine);
-    const float e = lane < r ? expf(mine - m) : 0.f;
-    const float lse = m + logf(warp_sum(e));
-    if (lane < r) logw[static_cast<size_t>(i) * r + lane] = mine - lse;
-  }
-}
-
-// Mixture epilogue (last line of Eq. 9).  One block per position; warps share the
-// n*r heads, then warp 0 mixes the experts (lane = expert).
+// Gate (Eq. 7) and mixture epilogue (last line of Eq. 9) in one launch.  One block
+// per position.  Phase 1: warps share the r experts, g[a] = W_g[a] . h[i], then
+// logw = log softmax(g).  Phase 2: warps share the n*r heads,
 //   lse[i,k]  = two-pass merge of the per-split (max, sum-exp) partials
 //   tgt[i,k]  = sum of the per-64-column target-logit partials
+// Phase 3 (warp 0, lane = expert):
 //   a[i,al]   = logw[i,al] + sum_s (tgt - lse)[i, s*r+al]
 //   logp[i]   = logsumexp_al a;  q = exp(a - logp)
-// Optionally the prefix scores logsumexp_al(logw + sum_{t<=s} C) for every s.
-__global__ void mixture_kernel(const float* __restrict__ part_m, const float* __restrict__ part_l,
-                               int splits, const float* __restrict__ tgt_part, int tgt_parts,
-                               const float* __restrict__ logw, float* __restrict__ lse_out,
-                               float* __restrict__ tgt_out, float* __restrict__ q_out,
-                               float* __restrict__ logp, float* __restrict__ logp_prefix, int N, int n,
-                               int r) {
+// and optionally the prefix scores logsumexp_al(logw + sum_{t<=s} C) for every s.
+__global__ void gate_mixture_kernel(const uint16_t* __restrict__ h, const uint16_t* __restrict__ W_g, int d,
+                                    const float* __restrict__ part_m, const float* __restrict__ part_l,
+                                    int splits, const float* __restrict__ tgt_part, int tgt_parts,
+                                    float* __restrict__ logw_out, float* __restrict__ lse_out,
+                                    float* __restrict__ tgt_out, float* __restrict__ q_out,
+                                    float* __restrict__ logp, float* __restrict__ logp_prefix, int N, int n,
+                                    int r) {
   __shared__ float c_s[CPMTP_MAX_N * CPMTP_MAX_R];
+  __shared__ float g_s[CPMTP_MAX_R];
   const int i = blockIdx.x;
   const int warp = threadIdx.x >> 5;
   const int nwarps = blockDim.x >> 5;
   const int lane = threadIdx.x & 31;
   const int K = n * r;
+  // phase 1: gate logits
+  {
+    const uint4* hrow = reinterpret_cast<const uint4*>(h + static_cast<size_t>(i) * d);
+    const int vecs = d >> 3;
+    for (int a = warp; a < r; a += nwarps) {
+      const uint4* wrow = reinterpret_cast<const uint4*>(W_g + static_cast<size_t>(a) * d);
+      float acc = 0.f;
+      for (int j = lane; j < vecs; j += 32) {
+        const uint4 hv = __ldg(hrow + j);
+        const uint4 wv = __ldg(wrow + j);
+        acc = fmaf(ptx::bf16_lo(hv.x), ptx::bf16_lo(wv.x), acc);
+        acc = fmaf(ptx::bf16_hi(hv.x), ptx::bf16_hi(wv.x), acc);
+        acc = fmaf(ptx::bf16_lo(hv.y), ptx::bf16_lo(wv.y), acc);
+        acc = fmaf(ptx::bf16_hi(hv.y), ptx::bf16_hi(wv.y), acc);
+        acc = fmaf(ptx::bf16_lo(hv.z), ptx::bf16_lo(wv.z), acc);
+        acc = fmaf(ptx::bf16_hi(hv.z), ptx::bf16_hi(wv.z), acc);
+        acc = fmaf(ptx::bf16_lo(hv.w), ptx::bf16_lo(wv.w), acc);
+        acc = fmaf(ptx::bf16_hi(hv.w), ptx::bf16_hi(wv.w), acc);
+      }
+      acc = warp_sum(acc);
+      if (lane == 0) g_s[a] = acc;
+    }
+  }
+  // phase 2: per-head vocabulary logsumexp and target logit
   for (int k = warp; k < K; k += nwarps) {
     const size_t row = static_cast<size_t>(i) * K + k;
-    // pass 1: global max over splits; pass 2: rescaled sum
     float m = -INFINITY;
     for (int j = lane; j < splits; j += 32) m = fmaxf(m, part_m[row * splits + j]);
     m = warp_max(m);
@@ -98,7 +89,15 @@ __global__ void mixture_kernel(const float* __restrict__ part_m, const float* __
   }
   __syncthreads();
   if (warp != 0) return;
-  float a = lane < r ? logw[static_cast<size_t>(i) * r + lane] : -INFINITY;
+  // phase 3: gate softmax and expert mixture
+  float a;
+  {
+    const float mine = lane < r ? g_s[lane] : -INFINITY;
+    const float m = warp_max(mine);
+    const float e = lane < r ? expf(mine - m) : 0.f;
+    a = mine - (m + logf(warp_sum(e)));
+    if (lane < r) logw_out[static_cast<size_t>(i) * r + lane] = a;
+  }
   for (int s = 0; s < n; ++s) {
     if (lane < r) a += c_s[s * r + lane];
     if (logp_prefix != nullptr || s == n - 1) {

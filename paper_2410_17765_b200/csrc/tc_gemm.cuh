@@ -76,13 +76,19 @@ __device__ __forceinline__ bool decode_unit(const Sched& s, int u, int& m_tile, 
   return n_end > n_begin;
 }
 
-template <int BN_, int STAGES_, bool A_MN_, bool B_MN_>
+// A_ROWS < 128 ("skinny A", K-major A only): the problem has at most A_ROWS rows, so only
+// that many rows of the A tile are fetched and given shared memory; the MMA still spans 128
+// rows and the accumulator rows beyond A_ROWS hold garbage that no epilogue may use.  The
+// space saved buys deeper pipelining of the B stream (bandwidth-bound draft scoring).
+template <int BN_, int STAGES_, bool A_MN_, bool B_MN_, int A_ROWS_ = kBM>
 struct TileCfg {
   static constexpr int BN = BN_;
   static constexpr int STAGES = STAGES_;
   static constexpr bool A_MN = A_MN_;
   static constexpr bool B_MN = B_MN_;
-  static constexpr int A_BYTES = kBM * kBK * 2;
+  static constexpr int A_ROWS = A_ROWS_;
+  static constexpr int A_BYTES = A_ROWS * kBK * 2;
+  static_assert(A_ROWS == kBM || (!A_MN_ && A_ROWS % 8 == 0 && A_ROWS >= 8), "skinny A needs a K-major A");
   static constexpr int B_BYTES = BN * kBK * 2;
   static constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
   static constexpr int TMEM_COLS = (2 * BN <= 32) ? 32 : (2 * BN <= 64) ? 64 : (2 * BN <= 128) ? 128
