@@ -41,6 +41,7 @@ WORKLOADS = {
 # captures summarised under profiles/ (None until captured, or once the kernel has changed since).
 NCU_TRAFFIC_BYTES = {
     "train_fwd": 1.211704e9 + 6.09024e6,   # profiles/lse_train_fwd.md
+    "decode_1": 1.051697e9 + 3.96288e6,    # profiles/decode_1.md
 }
 
 
