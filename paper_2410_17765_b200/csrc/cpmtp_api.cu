@@ -22,6 +22,9 @@ constexpr size_t kAlign = 256;
 constexpr size_t kLogitGradBudgetBytes = 4ull << 30;   // bound on the recomputed-logit-gradient chunk
 
 using CfgKK = TileCfg<kBN, kStages, false, false>;   // A K-major, B K-major
+constexpr int kWideStages = 3;                        // 64 KB per slot
+constexpr int kWideBM = 2 * kBM;
+using WideKK = TileCfg<kBN, kWideStages, false, false, kBM, 2>;   // 256 x 256 tiles, two row blocks share B
 using CfgKKSkinny = TileCfg<kBN, 5, false, false, 32>;   // <= 32 rows of A: bandwidth-bound draft scoring
 using CfgKM = TileCfg<kBN, kStages, false, true>;    // A K-major, B MN-major
 using CfgMM = TileCfg<kBN, kStages, true, true>;     // both MN-major
@@ -61,16 +64,23 @@ int validate_shape(const cpmtp_shape* s) {
 
 inline bool aligned(const void* p, size_t a) { return (reinterpret_cast<uintptr_t>(p) % a) == 0; }
 
+// Wide (256-row) tiles move a third fewer operand bytes per flop but cannot overlap their
+// epilogue with the next tile's MMAs, so they pay when the contraction is long enough to
+// amortise it; otherwise 128-row tiles with the double-buffered accumulator are used.
+bool use_wide(long long rows, long long kdim) { return rows >= 2 * kWideBM && kdim >= 4096; }
+
 // Column-split schedule of the fused unembedding: `group` row tiles x `splits`
 // vocabulary ranges run concurrently, so the rows' z tiles stay L2-resident while
 // each range of E is streamed once per group.  The split count minimises a simple
 // time model: max(makespan of the tensor work, HBM traffic / bandwidth); ties go
 // to the choice that keeps more SMs busy, then to fewer splits.
-Sched sched_lse(int m_tiles, int n_tiles, int M, int V, int d, int bn, int sms) {
+Sched sched_lse(int m_tiles, int n_tiles, int M, int V, int d, int bm, int slots) {
   // keep the concurrently swept z tiles (group * 128 rows * d * 2 B) within ~64 MB of L2
-  int max_group = static_cast<int>((64ll << 20) / (256ll * d));
+  // (bm = rows per row tile: 128 or 256; slots = tiles in flight = SMs)
+  const int sms = slots;
+  int max_group = static_cast<int>((64ll << 20) / (2ll * bm * d));
   if (max_group < 1) max_group = 1;
-  const double tile_t = 2.0 * kBM * bn * d / (1.4e15 / sms);
+  const double tile_t = 2.0 * bm * kBN * d / (1.4e15 / 148.0);
   int best_s = 1, best_ctas = 0;
   double best_score = -1.0;
   const int s_max = n_tiles < sms ? n_tiles : sms;
@@ -97,15 +107,18 @@ struct FwdLayout {
   size_t logw, q, wbar, lse, tgt, z, tgt_part, part_m, part_l, total;
   Sched lse_sched;
   int K, M;   // heads, rows of the unembedding GEMM
+  bool wide;  // the unembedding runs on 256-row tiles
 };
 
 FwdLayout fwd_layout(const cpmtp_shape& s, int sms) {
   FwdLayout L;
   L.K = s.n * s.r;
   L.M = s.N * L.K;
-  const int m_tiles = (L.M + kBM - 1) / kBM;
+  L.wide = use_wide(L.M, s.d);
+  const int bm = L.wide ? kWideBM : kBM;
+  const int m_tiles = (L.M + bm - 1) / bm;
   const int n_tiles = (s.V + kBN - 1) / kBN;
-  L.lse_sched = sched_lse(m_tiles, n_tiles, L.M, s.V, s.d, kBN, sms);
+  L.lse_sched = sched_lse(m_tiles, n_tiles, L.M, s.V, s.d, bm, sms);
   size_t off = 0;
   auto take = [&](size_t bytes) { size_t o = off; off = align_up(off + bytes); return o; };
   L.logw = take(sizeof(float) * s.N * s.r);
@@ -186,7 +199,7 @@ cudaError_t launch_gemm(const void* A, uint64_t a_rows, uint64_t a_ld, const voi
                         int* dev_status, int sms, cudaStream_t stream) {
   static bool attr_set[64] = {};
   CUtensorMap tA, tB;
-  if (!make_operand_tmap(&tA, A, Cfg::A_MN, a_rows, kdim, a_ld, Cfg::A_ROWS)) return cudaErrorInvalidValue;
+  if (!make_operand_tmap(&tA, A, Cfg::A_MN, a_rows, kdim, a_ld, Cfg::A_ROWS * Cfg::MB)) return cudaErrorInvalidValue;
   if (!make_operand_tmap(&tB, B, Cfg::B_MN, b_rows, kdim, b_ld, Cfg::BN)) return cudaErrorInvalidValue;
   constexpr int smem = gemm_smem_bytes<Cfg, Epi>();
   int dev = 0;
@@ -197,8 +210,28 @@ cudaError_t launch_gemm(const void* A, uint64_t a_rows, uint64_t a_ld, const voi
     attr_set[dev] = true;
   }
   const int grid = sched.units < sms ? sched.units : sms;
-  tc_gemm_kernel<Cfg, Epi><<<grid, kGemmThreads, smem, stream>>>(tA, tB, sched, ep, dev_status);
+  tc_gemm_kernel<Cfg, Epi><<<grid, Cfg::THREADS, smem, stream>>>(tA, tB, sched, ep, dev_status);
   return cudaGetLastError();
+}
+
+// A plain GEMM D[m_rows, n_cols] = A * B^T over `kdim`, every column tile its own unit, row tiles
+// swept in groups of about `group_rows` rows; wide tiles when the problem is large enough.
+template <bool A_MN, bool B_MN, class Epi>
+cudaError_t gemm_auto(const void* A, uint64_t a_ld, const void* B, uint64_t b_ld, long long m_rows, int n_cols,
+                      long long kdim, int group_rows, const typename Epi::Params& ep, int* dev_status, int sms,
+                      cudaStream_t stream) {
+  const int n_tiles = (n_cols + kBN - 1) / kBN;
+  const int k_blocks = static_cast<int>((kdim + kBK - 1) / kBK);
+  if (use_wide(m_rows, kdim)) {
+    const int m_tiles = static_cast<int>((m_rows + kWideBM - 1) / kWideBM);
+    const Sched sc = make_sched(m_tiles, n_tiles, n_tiles, group_rows / kWideBM, k_blocks);
+    return launch_gemm<TileCfg<kBN, kWideStages, A_MN, B_MN, kBM, 2>, Epi>(A, m_rows, a_ld, B, n_cols, b_ld, kdim, sc,
+                                                                           ep, dev_status, sms, stream);
+  }
+  const int m_tiles = static_cast<int>((m_rows + kBM - 1) / kBM);
+  const Sched sc = make_sched(m_tiles, n_tiles, n_tiles, group_rows / kBM, k_blocks);
+  return launch_gemm<TileCfg<kBN, kStages, A_MN, B_MN>, Epi>(A, m_rows, a_ld, B, n_cols, b_ld, kdim, sc, ep,
+                                                            dev_status, sms, stream);
 }
 
 #define CPMTP_TRY(expr)                         \
@@ -226,14 +259,13 @@ int run_forward(const cpmtp_shape& s, const uint16_t* h, const uint16_t* W_head,
   // head projection: z[N, K*d] = h[N, d] * W_cat[K*d, d]^T, plus the fp32 target-logit partials
   {
     ProfScope prof(CPMTP_STAGE_PROJ, stream);
-    const int m_tiles = (s.N + kBM - 1) / kBM;
-    const int n_tiles = (ncols + kBN - 1) / kBN;
-    const Sched sc = make_sched(m_tiles, n_tiles, n_tiles, m_tiles < 64 ? m_tiles : 64, s.d / kBK);
     EpiProj<kBN>::Params ep{z, tgt_part, E, x, dev_status, s.N, ncols, s.d, s.V, s.n, s.r};
     if (s.N <= CfgKKSkinny::A_ROWS) {
+      const int n_tiles = (ncols + kBN - 1) / kBN;
+      const Sched sc = make_sched(1, n_tiles, n_tiles, 1, s.d / kBK);
       CPMTP_TRY((launch_gemm<CfgKKSkinny, EpiProj<kBN>>(h, s.N, s.d, W_head, ncols, s.d, s.d, sc, ep, dev_status, sms, stream)));
     } else {
-      CPMTP_TRY((launch_gemm<CfgKK, EpiProj<kBN>>(h, s.N, s.d, W_head, ncols, s.d, s.d, sc, ep, dev_status, sms, stream)));
+      CPMTP_TRY((gemm_auto<false, false, EpiProj<kBN>>(h, s.d, W_head, s.d, s.N, ncols, s.d, 8192, ep, dev_status, sms, stream)));
     }
   }
   // unembedding fused with the vocabulary log-sum-exp (Eq. 6, Eq. 8)
@@ -242,6 +274,8 @@ int run_forward(const cpmtp_shape& s, const uint16_t* h, const uint16_t* W_head,
     EpiLse<kBN>::Params ep{part_m, part_l, L.M, s.V, L.lse_sched.n_splits};
     if (L.M <= CfgKKSkinny::A_ROWS) {
       CPMTP_TRY((launch_gemm<CfgKKSkinny, EpiLse<kBN>>(z, L.M, s.d, E, s.V, s.d, s.d, L.lse_sched, ep, dev_status, sms, stream)));
+    } else if (L.wide) {
+      CPMTP_TRY((launch_gemm<WideKK, EpiLse<kBN>>(z, L.M, s.d, E, s.V, s.d, s.d, L.lse_sched, ep, dev_status, sms, stream)));
     } else {
       CPMTP_TRY((launch_gemm<CfgKK, EpiLse<kBN>>(z, L.M, s.d, E, s.V, s.d, s.d, L.lse_sched, ep, dev_status, sms, stream)));
     }
@@ -508,28 +542,23 @@ int cpmtp_backward(const cpmtp_shape* shape, const void* h, const void* W_head, 
     {
       ProfScope prof(CPMTP_STAGE_LOGIT_GRAD, st);
       EpiLogitGrad<kBN>::Params ep{G, saved->lse, coef, x, row0, rows, L.ldg, V, K, s.n, s.r};
-      const int n_tiles = (L.ldg + kBN - 1) / kBN;
-      const Sched sc = make_sched(m_tiles, n_tiles, n_tiles, 16, d / kBK);
-      CPMTP_TRY((launch_gemm<CfgKK, EpiLogitGrad<kBN>>(zc, rows, d, Eb, V, d, d, sc, ep, dev_status, sms, st)));
+      CPMTP_TRY((gemm_auto<false, false, EpiLogitGrad<kBN>>(zc, d, Eb, d, rows, V, d, 2048, ep, dev_status, sms, st)));
     }
     // dz[rows, d] = G[rows, V] * E[V, d]
     {
       ProfScope prof(CPMTP_STAGE_DZ, st);
       EpiStoreBf16<kBN, false>::Params ep{dz + row0 * d, nullptr, nullptr, rows, d, d, 0};
-      const Sched sc = make_sched(m_tiles, d_tiles, d_tiles, 16, (V + kBK - 1) / kBK);
-      CPMTP_TRY((launch_gemm<CfgKM, EpiStoreBf16<kBN, false>>(G, rows, L.ldg, Eb, d, d, V, sc, ep, dev_status, sms, st)));
+      CPMTP_TRY((gemm_auto<false, true, EpiStoreBf16<kBN, false>>(G, L.ldg, Eb, d, rows, d, V, 2048, ep, dev_status, sms, st)));
     }
     // dE[V, d] (+)= G^T[V, rows] * z[rows, d]
     {
       ProfScope prof(CPMTP_STAGE_DE, st);
-      const int v_tiles = (V + kBM - 1) / kBM;
-      const Sched sc = make_sched(v_tiles, d_tiles, d_tiles, 16, (rows + kBK - 1) / kBK);
       if (L.chunks == 1) {
         EpiStoreBf16<kBN, false>::Params ep{static_cast<uint16_t*>(dE), nullptr, nullptr, V, d, d, 0};
-        CPMTP_TRY((launch_gemm<CfgMM, EpiStoreBf16<kBN, false>>(G, V, L.ldg, zc, d, d, rows, sc, ep, dev_status, sms, st)));
+        CPMTP_TRY((gemm_auto<true, true, EpiStoreBf16<kBN, false>>(G, L.ldg, zc, d, V, d, rows, 2048, ep, dev_status, sms, st)));
       } else {
         EpiAccumF32<kBN>::Params ep{dE32, V, d, d, c > 0 ? 1 : 0};
-        CPMTP_TRY((launch_gemm<CfgMM, EpiAccumF32<kBN>>(G, V, L.ldg, zc, d, d, rows, sc, ep, dev_status, sms, st)));
+        CPMTP_TRY((gemm_auto<true, true, EpiAccumF32<kBN>>(G, L.ldg, zc, d, V, d, rows, 2048, ep, dev_status, sms, st)));
       }
     }
   }
@@ -542,17 +571,13 @@ int cpmtp_backward(const cpmtp_shape* shape, const void* h, const void* W_head, 
   {
     ProfScope prof(CPMTP_STAGE_DW_HEAD, st);
     EpiStoreBf16<kBN, false>::Params ep{static_cast<uint16_t*>(dW_head), nullptr, nullptr, ncols, d, d, 0};
-    const int m_tiles = (ncols + kBM - 1) / kBM;
-    const Sched sc = make_sched(m_tiles, d_tiles, d_tiles, 16, (s.N + kBK - 1) / kBK);
-    CPMTP_TRY((launch_gemm<CfgMM, EpiStoreBf16<kBN, false>>(dz, ncols, ncols, h, d, d, s.N, sc, ep, dev_status, sms, st)));
+    CPMTP_TRY((gemm_auto<true, true, EpiStoreBf16<kBN, false>>(dz, ncols, h, d, ncols, d, s.N, 2048, ep, dev_status, sms, st)));
   }
   // dh[N, d] = dz[N, K*d] * W_cat[K*d, d] + dg * W_g
   {
     ProfScope prof(CPMTP_STAGE_DH, st);
     EpiStoreBf16<kBN, true>::Params ep{static_cast<uint16_t*>(dh), dg, static_cast<const uint16_t*>(W_g), s.N, d, d, s.r};
-    const int m_tiles = (s.N + kBM - 1) / kBM;
-    const Sched sc = make_sched(m_tiles, d_tiles, d_tiles, 16, ncols / kBK);
-    CPMTP_TRY((launch_gemm<CfgKM, EpiStoreBf16<kBN, true>>(dz, s.N, ncols, W_head, d, d, ncols, sc, ep, dev_status, sms, st)));
+    CPMTP_TRY((gemm_auto<false, true, EpiStoreBf16<kBN, true>>(dz, ncols, W_head, d, s.N, d, ncols, 2048, ep, dev_status, sms, st)));
   }
   // dW_g[r, d] = dg^T * h
   {

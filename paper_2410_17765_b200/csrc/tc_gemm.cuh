@@ -2,13 +2,18 @@
 //
 //   D[M, N] = A[M, K] * B[N, K]^T      bf16 operands, fp32 accumulation in TMEM
 //
-// One CTA per SM, 192 threads:
+// One CTA per SM, 64 + 128*MB threads:
 //   warp 0      TMA producer (one lane): global -> 128B-swizzled shared tiles
 //   warp 1      MMA issuer (one lane): tcgen05.mma, accumulators in TMEM
-//   warps 2..5  epilogue: tcgen05.ld the 128 x BN fp32 tile and hand it to `Epi`
-// The accumulator is double-buffered in TMEM (2 x BN columns) so the epilogue of
-// tile j overlaps the MMAs of tile j+1.  The shared-memory ring has STAGES slots
-// of (128 x 64) A + (BN x 64) B.
+//   then 4 epilogue warps per 128-row block: tcgen05.ld the 128 x BN fp32 block and
+//   hand it to `Epi`
+// MB = 1: a 128 x BN tile, accumulator double-buffered in TMEM (2 x BN columns) so the
+//   epilogue of tile j overlaps the MMAs of tile j+1; ring slots of (128 x 64) A + (BN x 64) B.
+// MB = 2 ("wide"): a 256 x 256 tile as two 128-row blocks that share every B slot (two MMAs
+//   per K step), filling all 512 TMEM columns, so the epilogue is not overlapped.  Operand
+//   bytes moved from L2 into the SM per flop drop by a third (64 KB per 256x256x64 instead
+//   of 48 KB per 128x256x64); measured on B200 that traffic, not the tensor pipe, bounds the
+//   sustained rate (under the power cap as well as at full clocks), so the trade pays.
 //
 // Either operand may be "K-major" (contraction index contiguous in global
 // memory: the tensor map's inner dimension is K) or "MN-major" (the M or N index
@@ -29,8 +34,7 @@ namespace cpmtp {
 
 constexpr int kBM = 128;          // rows per tile = TMEM lanes
 constexpr int kBK = 64;           // bf16 elements per 128-byte swizzle row
-constexpr int kGemmThreads = 192;
-constexpr int kEpiThreads = 128;
+constexpr int kEpiThreads = 128;   // epilogue threads per 128-row block
 
 // Values raised in the device status word.
 constexpr int kDevOk = 0;
@@ -38,7 +42,7 @@ constexpr int kDevTargetOutOfRange = 1;
 constexpr int kDevWaitTimeout = 2;
 
 struct Sched {
-  int m_tiles;    // number of 128-row tiles
+  int m_tiles;    // number of (128 * MB)-row tiles
   int n_tiles;    // number of BN-column tiles
   int n_splits;   // column tiles are cut into this many contiguous ranges
   int m_group;    // row tiles that are swept together (L2 locality)
@@ -80,19 +84,28 @@ __device__ __forceinline__ bool decode_unit(const Sched& s, int u, int& m_tile, 
 // that many rows of the A tile are fetched and given shared memory; the MMA still spans 128
 // rows and the accumulator rows beyond A_ROWS hold garbage that no epilogue may use.  The
 // space saved buys deeper pipelining of the B stream (bandwidth-bound draft scoring).
-template <int BN_, int STAGES_, bool A_MN_, bool B_MN_, int A_ROWS_ = kBM>
+template <int BN_, int STAGES_, bool A_MN_, bool B_MN_, int A_ROWS_ = kBM, int MB_ = 1>
 struct TileCfg {
   static constexpr int BN = BN_;
   static constexpr int STAGES = STAGES_;
   static constexpr bool A_MN = A_MN_;
   static constexpr bool B_MN = B_MN_;
-  static constexpr int A_ROWS = A_ROWS_;
-  static constexpr int A_BYTES = A_ROWS * kBK * 2;
+  static constexpr int MB = MB_;                       // 128-row blocks per tile
+  static constexpr int A_ROWS = A_ROWS_;               // rows of A fetched per 128-row block
+  static constexpr int TILE_M = kBM * MB;
+  static constexpr int A_BLOCK_BYTES = A_ROWS * kBK * 2;
+  static constexpr int A_BYTES = A_BLOCK_BYTES * MB;
+  static constexpr int ACC_STAGES = MB == 1 ? 2 : 1;
+  static constexpr int THREADS = 64 + kEpiThreads * MB;
+  static_assert(MB == 1 || MB == 2, "one or two 128-row blocks");
+  static_assert(MB == 1 || (A_ROWS == kBM && BN == 256), "wide tiles are 256 x 256");
   static_assert(A_ROWS == kBM || (!A_MN_ && A_ROWS % 8 == 0 && A_ROWS >= 8), "skinny A needs a K-major A");
   static constexpr int B_BYTES = BN * kBK * 2;
   static constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
-  static constexpr int TMEM_COLS = (2 * BN <= 32) ? 32 : (2 * BN <= 64) ? 64 : (2 * BN <= 128) ? 128
-                                   : (2 * BN <= 256) ? 256 : 512;
+  static constexpr int ACC_COLS = BN * MB * ACC_STAGES;
+  static constexpr int TMEM_COLS = (ACC_COLS <= 32) ? 32 : (ACC_COLS <= 64) ? 64 : (ACC_COLS <= 128) ? 128
+                                   : (ACC_COLS <= 256) ? 256 : 512;
+  static_assert(ACC_COLS <= 512, "TMEM has 512 columns");
   static_assert(BN % 16 == 0 && BN >= 16 && BN <= 256, "MMA N must be a multiple of 16 in [16, 256]");
   static_assert(!B_MN || BN % 64 == 0, "an MN-major B tile is loaded in 64-wide boxes");
   static_assert(STAGE_BYTES % 1024 == 0, "stages must keep 1024-byte alignment for the swizzle");
@@ -106,7 +119,7 @@ constexpr int gemm_smem_bytes() {
 }
 
 template <class Cfg, class Epi>
-__global__ void __launch_bounds__(kGemmThreads, 1)
+__global__ void __launch_bounds__(Cfg::THREADS, 1)
 tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
                const Sched sched, const typename Epi::Params ep, int* __restrict__ dev_status) {
   extern __shared__ uint8_t smem_raw[];
@@ -137,7 +150,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     }
     for (int a = 0; a < 2; ++a) {
       ptx::mbar_init(tfull_bar(a), 1);
-      ptx::mbar_init(tempty_bar(a), kEpiThreads);
+      ptx::mbar_init(tempty_bar(a), kEpiThreads * Cfg::MB);
     }
     ptx::mbar_init(drain_bar, 1);
     *abort_flag = 0;
@@ -171,11 +184,12 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             const uint32_t a_dst = tiles_addr + s * Cfg::STAGE_BYTES;
             const uint32_t b_dst = a_dst + Cfg::A_BYTES;
             if constexpr (!Cfg::A_MN) {
-              ptx::tma_load_2d(a_dst, &tmA, full_bar(s), kb * kBK, m_tile * kBM);
+              // one box of A_ROWS * MB rows: block b lands at a_dst + b * A_BLOCK_BYTES
+              ptx::tma_load_2d(a_dst, &tmA, full_bar(s), kb * kBK, m_tile * Cfg::TILE_M);
             } else {
 #pragma unroll
-              for (int j = 0; j < kBM / 64; ++j)
-                ptx::tma_load_2d(a_dst + j * 8192, &tmA, full_bar(s), m_tile * kBM + j * 64, kb * kBK);
+              for (int j = 0; j < Cfg::TILE_M / 64; ++j)
+                ptx::tma_load_2d(a_dst + j * 8192, &tmA, full_bar(s), m_tile * Cfg::TILE_M + j * 64, kb * kBK);
             }
             if constexpr (!Cfg::B_MN) {
               ptx::tma_load_2d(b_dst, &tmB, full_bar(s), kb * kBK, nt * Cfg::BN);
@@ -210,11 +224,11 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         int m_tile, split, n_begin, n_end;
         if (!decode_unit(sched, u, m_tile, split, n_begin, n_end)) continue;
         for (int nt = n_begin; nt < n_end && alive; ++nt, ++acc_it) {
-          const int acc = acc_it & 1;
-          const uint32_t acc_ph = (acc_it >> 1) & 1;
+          const int acc = acc_it % Cfg::ACC_STAGES;
+          const uint32_t acc_ph = (acc_it / Cfg::ACC_STAGES) & 1;
           if (!ptx::mbar_wait(tempty_bar(acc), acc_ph ^ 1u, abort_flag)) { alive = false; break; }
           ptx::tc_fence_after_sync();
-          const uint32_t d_tmem = tmem_base + acc * Cfg::BN;
+          const uint32_t d_tmem = tmem_base + acc * Cfg::BN * Cfg::MB;
           for (int kb = 0; kb < sched.k_blocks; ++kb, ++it) {
             const int s = it % Cfg::STAGES;
             const uint32_t ph = (it / Cfg::STAGES) & 1;
@@ -224,9 +238,13 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             const uint32_t b_src = a_src + Cfg::A_BYTES;
 #pragma unroll
             for (int kk = 0; kk < kBK / 16; ++kk) {
-              const uint64_t adesc = ptx::make_smem_desc_sw128(a_src + kk * a_kstep, a_lbo, 1024);
               const uint64_t bdesc = ptx::make_smem_desc_sw128(b_src + kk * b_kstep, b_lbo, 1024);
-              ptx::umma_bf16(d_tmem, adesc, bdesc, idesc, (kb | kk) != 0 ? 1u : 0u);
+#pragma unroll
+              for (int mb = 0; mb < Cfg::MB; ++mb) {
+                const uint64_t adesc =
+                    ptx::make_smem_desc_sw128(a_src + mb * Cfg::A_BLOCK_BYTES + kk * a_kstep, a_lbo, 1024);
+                ptx::umma_bf16(d_tmem + mb * Cfg::BN, adesc, bdesc, idesc, (kb | kk) != 0 ? 1u : 0u);
+              }
             }
             ptx::umma_commit(empty_bar(s));   // frees the slot once these MMAs have read it
           }
@@ -243,26 +261,29 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     // same barrier, so they either all pass or all time out, and no warp is left
     // alone at a barrier an epilogue might use internally.
     const int quarter = warp & 3;                 // TMEM lane quarter this warp may read
-    const int row_in_tile = quarter * 32 + lane;
-    const int epi_tid = threadIdx.x - 64;
+    const int mblock = (warp - 2) >> 2;           // which 128-row block of the tile
+    const int row_in_tile = quarter * 32 + lane;  // row within that block
+    const int epi_tid = (threadIdx.x - 64) & (kEpiThreads - 1);
     typename Epi::State st;
     int acc_it = 0;
     bool alive = true;
     for (int u = blockIdx.x; u < sched.units && alive; u += gridDim.x) {
       int m_tile, split, n_begin, n_end;
       if (!decode_unit(sched, u, m_tile, split, n_begin, n_end)) continue;
-      Epi::unit_begin(ep, st, m_tile, split, row_in_tile);
+      const int m_block_tile = m_tile * Cfg::MB + mblock;   // index of this warp's 128-row block
+      Epi::unit_begin(ep, st, m_block_tile, split, row_in_tile);
       for (int nt = n_begin; nt < n_end; ++nt, ++acc_it) {
-        const int acc = acc_it & 1;
-        const uint32_t acc_ph = (acc_it >> 1) & 1;
+        const int acc = acc_it % Cfg::ACC_STAGES;
+        const uint32_t acc_ph = (acc_it / Cfg::ACC_STAGES) & 1;
         if (!ptx::mbar_wait(tfull_bar(acc), acc_ph, abort_flag, false)) { alive = false; break; }
         ptx::tc_fence_after_sync();
-        const uint32_t tacc = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16) + acc * Cfg::BN;
-        Epi::tile(ep, st, tacc, m_tile, nt, row_in_tile, epi_smem, epi_tid);
+        const uint32_t tacc = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16) +
+                              (acc * Cfg::MB + mblock) * Cfg::BN;
+        Epi::tile(ep, st, tacc, m_block_tile, nt, row_in_tile, epi_smem, epi_tid);
         ptx::tc_fence_before_sync();
         ptx::mbar_arrive(tempty_bar(acc));
       }
-      if (alive) Epi::unit_end(ep, st, m_tile, split, row_in_tile, epi_smem, epi_tid);
+      if (alive) Epi::unit_end(ep, st, m_block_tile, split, row_in_tile, epi_smem, epi_tid);
     }
   }
 
