@@ -78,7 +78,12 @@ Sched sched_lse(int m_tiles, int n_tiles, int M, int V, int d, int bm, int slots
   // keep the concurrently swept z tiles (group * 128 rows * d * 2 B) within ~64 MB of L2
   // (bm = rows per row tile: 128 or 256; slots = tiles in flight = SMs)
   const int sms = slots;
-  int max_group = static_cast<int>((64ll << 20) / (2ll * bm * d));
+  long long l2_budget_mb = 64;
+  if (const char* env = std::getenv("CPMTP_LSE_GROUP_MB")) {   // tuning knob: L2 budget for the swept z tiles
+    const long long v = std::atoll(env);
+    if (v >= 1 && v <= 1024) l2_budget_mb = v;
+  }
+  int max_group = static_cast<int>((l2_budget_mb << 20) / (2ll * bm * d));
   if (max_group < 1) max_group = 1;
   const double tile_t = 2.0 * bm * kBN * d / (1.4e15 / 148.0);
   int best_s = 1, best_ctas = 0;
