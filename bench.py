@@ -34,6 +34,7 @@ WORKLOADS = {
     "decode_1": ("decode_1", "score", {}, None),
     "decode_8": ("decode_8", "score", {}, None),
     "decode_64": ("decode_64", "score", {}, None),
+    "train_fwd_bwd_small": ("train_fwd_bwd_small", "fwd_bwd", {}, None),
     "tiny": ("tiny", "fwd_bwd", {}, None),
 }
 

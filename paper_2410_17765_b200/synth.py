@@ -42,6 +42,8 @@ CONFIGS = {
     "decode_8": Shape(N=8, d=4096, V=128256, n=4, r=8),
     "decode_64": Shape(N=64, d=4096, V=128256, n=4, r=8),
     "bigvocab_fwd_bwd": Shape(N=8192, d=4096, V=128256, n=4, r=16),
+    # train_fwd_bwd at 1/16 of the positions: same kernels and tile shapes, small enough to profile
+    "train_fwd_bwd_small": Shape(N=512, d=4096, V=32000, n=4, r=8),
 }
 
 
