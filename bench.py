@@ -35,6 +35,7 @@ WORKLOADS = {
     "decode_8": ("decode_8", "score", {}, None),
     "decode_64": ("decode_64", "score", {}, None),
     "train_fwd_bwd_small": ("train_fwd_bwd_small", "fwd_bwd", {}, None),
+    "bigvocab_fwd_small": ("bigvocab_fwd_small", "fwd", {"targets": "zipf"}, 1.0),
     "tiny": ("tiny", "fwd_bwd", {}, None),
 }
 

@@ -75,10 +75,14 @@ bool use_wide(long long rows, long long kdim) { return rows >= 2 * kWideBM && kd
 // time model: max(makespan of the tensor work, HBM traffic / bandwidth); ties go
 // to the choice that keeps more SMs busy, then to fewer splits.
 Sched sched_lse(int m_tiles, int n_tiles, int M, int V, int d, int bm, int slots) {
-  // keep the concurrently swept z tiles (group * 128 rows * d * 2 B) within ~64 MB of L2
+  // keep the concurrently swept z tiles (group * bm rows * d * 2 B) within a budget of L2
   // (bm = rows per row tile: 128 or 256; slots = tiles in flight = SMs)
   const int sms = slots;
-  long long l2_budget_mb = 64;
+  // L2 budget for the z tiles a group keeps re-reading.  Measured with DRAM-byte counters on
+  // B200: with 256-row tiles at d = 4096 (2 MB per tile) 12 tiles x 12 vocabulary ranges gave the
+  // least DRAM traffic and the best time at V = 32000 and V = 128256; larger groups start to
+  // evict one another's z tiles and the E stream.  The 0.5 MB tiles at d = 2048 did best with 64 MB.
+  long long l2_budget_mb = bm > kBM ? 24 : 64;
   if (const char* env = std::getenv("CPMTP_LSE_GROUP_MB")) {   // tuning knob: L2 budget for the swept z tiles
     const long long v = std::atoll(env);
     if (v >= 1 && v <= 1024) l2_budget_mb = v;
@@ -103,6 +107,10 @@ Sched sched_lse(int m_tiles, int n_tiles, int M, int V, int d, int bm, int slots
       best_s = s;
       best_ctas = ctas;
     }
+  }
+  if (const char* env = std::getenv("CPMTP_LSE_SPLITS")) {   // tuning knob: force the split count
+    const int v = std::atoi(env);
+    if (v >= 1 && v <= s_max) best_s = v;
   }
   const int group = static_cast<long long>(m_tiles) * best_s >= sms ? (sms / best_s) : m_tiles;
   return make_sched(m_tiles, n_tiles, best_s, group < 1 ? 1 : group, d / kBK);

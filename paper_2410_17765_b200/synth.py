@@ -44,6 +44,8 @@ CONFIGS = {
     "bigvocab_fwd_bwd": Shape(N=8192, d=4096, V=128256, n=4, r=16),
     # train_fwd_bwd at 1/16 of the positions: same kernels and tile shapes, small enough to profile
     "train_fwd_bwd_small": Shape(N=512, d=4096, V=32000, n=4, r=8),
+    # bigvocab at 1/4 of the positions (forward only): same schedule regime, profilable
+    "bigvocab_fwd_small": Shape(N=2048, d=4096, V=128256, n=4, r=16),
 }
 
 

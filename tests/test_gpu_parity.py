@@ -36,6 +36,9 @@ CASES = {
     "ragged_stress": dict(shape=synth.Shape(N=37, d=192, V=777, n=3, r=5), weight_scale=8.0),
     "rank1": dict(shape=synth.Shape(N=130, d=128, V=300, n=4, r=1)),
     "wide": dict(shape=synth.Shape(N=300, d=512, V=2100, n=2, r=8), targets="zipf"),
+    "max_heads": dict(shape=synth.Shape(N=20, d=64, V=130, n=8, r=32)),
+    "single": dict(shape=synth.Shape(N=1, d=128, V=50, n=1, r=2)),
+    "long_k": dict(shape=synth.Shape(N=40, d=4096, V=600, n=2, r=8)),
 }
 
 
@@ -73,7 +76,7 @@ def test_forward_matches_oracle(name):
 
 
 @pytest.mark.parametrize("name,chunk_rows", [("tiny", None), ("tiny", 256), ("ragged", 128), ("ragged_stress", None),
-                                             ("rank1", None), ("wide", 1024)])
+                                             ("rank1", None), ("wide", 1024), ("max_heads", 512), ("single", None), ("long_k", None)])
 def test_backward_matches_oracle(name, chunk_rows):
     from paper_2410_17765_b200 import binding
 
