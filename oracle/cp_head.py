@@ -28,7 +28,9 @@ Readings of the paper taken here:
 
 Parity pins: every function below is pinned by tests/test_oracle_*.py
 (closed forms, brute-force normalisation, the rank-1 reduction to independent
-cross-entropies, finite differences).  Nothing here is "parity unpinned".
+cross-entropies, finite differences; for draft generation the brute-force
+conditionals of the full joint tensor and sampling frequencies).  Nothing here
+is "parity unpinned".
 """
 from __future__ import annotations
 
@@ -197,3 +199,62 @@ def backward(h, W_head, E, W_g, x, n: int, r: int, *, aux_coef: float = 0.0,
         dW_head[k] = dz.T @ hd
         dh += dz @ Wk
     return Gradients(dh=dh, dW_head=dW_head, dE=dE, dW_g=dW_g, dg=dg, c=c)
+
+
+@dataclass
+class Draft:
+    tokens: np.ndarray       # [N, n]      drafted tokens x_{t+1..t+n}
+    logp_joint: np.ndarray   # [N]         log P(tokens) under the CP head (Eq. 9 at the drafted tokens)
+    topk_tokens: np.ndarray  # [N, n, k]   most likely next tokens given the drafted prefix, best first
+    topk_logp: np.ndarray    # [N, n, k]   their conditional log-probabilities
+    mix: np.ndarray          # [N, n, V]   log P(x_{t+1..t+s-1} = drafted prefix, x_{t+s} = v)
+
+
+def draft(h, W_head, E, W_g, n: int, r: int, *, topk: int = 1, uniform=None,
+          temperature: float = 1.0) -> Draft:
+    """Sequential draft generation from the factors (sampling section).
+
+    The first token comes from the marginal of Eq. 11; for every later token the
+    expert weights are multiplied by the factors of the tokens already drawn
+    (b_alpha = w_alpha * prod_{t<s} P^(t)(x_t | alpha), the prose under Eq. 12)
+    and the next token is drawn from  sum_alpha b_alpha P^(s)(v | alpha) / sum_alpha b_alpha
+    (the printed Eq. 12 / Eq. 13 omit the s-th factor and the normaliser; this is the
+    reading their surrounding text describes).
+
+    uniform=None: temperature 0, the most likely token is taken (ties -> lowest id).
+    uniform [N, n, V] in (0, 1): the token is drawn exactly from the conditional
+    distribution, sharpened by 1/temperature, with the Gumbel-max rule
+    argmax_v( log p(v) / temperature - log(-log u[v]) ).
+    topk: the k most likely tokens of each conditional (unperturbed), best first.
+    """
+    hd, Ed = _f64(h), _f64(E)
+    N = hd.shape[0]
+    V = Ed.shape[0]
+    logw = gate_log_weights(h, W_g)
+    logP = np.empty((N, n, r, V))
+    for k in range(n * r):
+        s, alpha = divmod(k, r)
+        S = head_projection(hd, W_head[k]) @ Ed.T
+        logP[:, s, alpha, :] = S - logsumexp(S, axis=1)[:, None]
+    lb = logw.copy()                                   # log b_alpha
+    rows = np.arange(N)
+    tokens = np.empty((N, n), dtype=np.int64)
+    top_t = np.empty((N, n, topk), dtype=np.int64)
+    top_lp = np.empty((N, n, topk))
+    mixes = np.empty((N, n, V))
+    u = None if uniform is None else _f64(uniform)
+    for s in range(n):
+        mix = logsumexp(lb[:, :, None] + logP[:, s, :, :], axis=1)      # [N, V]
+        norm = logsumexp(lb, axis=1)                                    # log sum_alpha b_alpha
+        mixes[:, s, :] = mix
+        order = np.argsort(-mix, axis=1, kind="stable")[:, :topk]
+        top_t[:, s, :] = order
+        top_lp[:, s, :] = np.take_along_axis(mix, order, axis=1) - norm[:, None]
+        if u is None:
+            x_s = order[:, 0]
+        else:
+            x_s = np.argmax((mix - norm[:, None]) / temperature - np.log(-np.log(u[:, s, :])), axis=1)
+        tokens[:, s] = x_s
+        lb = lb + logP[rows, s, :, x_s]
+    return Draft(tokens=tokens, logp_joint=logsumexp(lb, axis=1), topk_tokens=top_t, topk_logp=top_lp,
+                 mix=mixes)

@@ -39,6 +39,7 @@ CASES = {
     "max_heads": dict(shape=synth.Shape(N=20, d=64, V=130, n=8, r=32)),
     "single": dict(shape=synth.Shape(N=1, d=128, V=50, n=1, r=2)),
     "long_k": dict(shape=synth.Shape(N=40, d=4096, V=600, n=2, r=8)),
+    "many_rows": dict(shape=synth.Shape(N=4096, d=1024, V=64, n=2, r=2)),
 }
 
 
@@ -76,7 +77,7 @@ def test_forward_matches_oracle(name):
 
 
 @pytest.mark.parametrize("name,chunk_rows", [("tiny", None), ("tiny", 256), ("ragged", 128), ("ragged_stress", None),
-                                             ("rank1", None), ("wide", 1024), ("max_heads", 512), ("single", None), ("long_k", None)])
+                                             ("rank1", None), ("wide", 1024), ("max_heads", 512), ("single", None), ("long_k", None), ("many_rows", None)])
 def test_backward_matches_oracle(name, chunk_rows):
     from paper_2410_17765_b200 import binding
 
