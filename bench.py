@@ -34,6 +34,7 @@ WORKLOADS = {
     "decode_1": ("decode_1", "score", {}, None),
     "decode_8": ("decode_8", "score", {}, None),
     "decode_64": ("decode_64", "score", {}, None),
+    "draft_8": ("decode_8", "sample", {}, None),
     "train_fwd_bwd_small": ("train_fwd_bwd_small", "fwd_bwd", {}, None),
     "bigvocab_fwd_small": ("bigvocab_fwd_small", "fwd", {"targets": "zipf"}, 1.0),
     "tiny": ("tiny", "fwd_bwd", {}, None),
@@ -192,6 +193,7 @@ def run_ours(args, rank: int, world: int, local_rank: int):
     status = torch.zeros(1, dtype=torch.int32, device="cuda")
     saved = binding.Saved.alloc(cs) if kind == "fwd_bwd" else None
     ws_bwd = binding.alloc_workspace(binding.workspace_bytes(cs, binding.OP_BACKWARD)) if kind == "fwd_bwd" else None
+    ws_smp = binding.alloc_workspace(binding.workspace_bytes(cs, binding.OP_SAMPLE)) if kind == "sample" else None
     out_f, out_b, out_s = {}, {}, {}
 
     def step():
@@ -202,6 +204,8 @@ def run_ours(args, rank: int, world: int, local_rank: int):
                             out=out_f)
             binding.backward(h, W_head, E, W_g, x, saved, aux_coef=aux, workspace=ws_bwd, dev_status=status,
                              out=out_b)
+        elif kind == "sample":
+            binding.sample_draft(h, W_head, E, W_g, shape.n, topk=5, workspace=ws_smp, dev_status=status, out=out_s)
         else:
             binding.score_draft(h, W_head, E, W_g, x, workspace=ws_fwd, dev_status=status, out=out_s)
 
@@ -209,7 +213,15 @@ def run_ours(args, rank: int, world: int, local_rank: int):
     logp_pin = torch.empty(shape.N, dtype=torch.float32).pin_memory()
     loss_pin = torch.empty(1, dtype=torch.float32).pin_memory()
 
+    draft_pin = torch.empty((shape.N, shape.n), dtype=torch.int32).pin_memory()
+
     def step_e2e():
+        if kind == "sample":
+            h.copy_(h_pin, non_blocking=True)
+            binding.sample_draft(h, W_head, E, W_g, shape.n, topk=5, workspace=ws_smp, dev_status=status, out=out_s)
+            draft_pin.copy_(out_s["draft"], non_blocking=True)
+            torch.cuda.current_stream().synchronize()
+            return
         binding.forward_host(h_pin, W_head, E, W_g, x_pin, logp_pin, loss_pin, aux_coef=aux, saved=saved,
                              workspace=ws_fwd, dev_status=status)
         if kind == "fwd_bwd":
@@ -259,7 +271,7 @@ def run_ours(args, rank: int, world: int, local_rank: int):
     dominant = "lse"
     dom_ms, dom_launches = stages.get(dominant, (0.0, 0))
     avg_ms = dom_ms / max(1, dom_launches)
-    if kind == "score" and shape.N * K * 2 < 250:   # below the ridge: HBM-bound streaming of E
+    if kind in ("score", "sample") and shape.N * K * 2 < 250:   # below the ridge: HBM-bound streaming of E
         alg = 2.0 * shape.V * shape.d
         roof = {"bound": "hbm", "achieved": alg / (avg_ms * 1e-3) / 1e9, "peak": peaks["hbm_gbs"], "unit": "GB/s"}
     else:
@@ -285,8 +297,10 @@ def run_ours(args, rank: int, world: int, local_rank: int):
                    "targets": extra.get("targets", "uniform"), "l2": "inputs larger than L2 (no flush)",
                    "per_gpu_positions": shape.N},
         "clocks": clocks,
-        "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": shape.N * shape.d * 2 + shape.N * shape.n * 4,
-                "d2h_bytes_per_step": shape.N * 4 + 4, "ms_per_step": ms_e2e / args.steps},
+        "e2e": {"value": e2e_value, "unit": UNIT,
+                "h2d_bytes_per_step": shape.N * shape.d * 2 + (0 if kind == "sample" else shape.N * shape.n * 4),
+                "d2h_bytes_per_step": shape.N * shape.n * 4 if kind == "sample" else shape.N * 4 + 4,
+                "ms_per_step": ms_e2e / args.steps},
         "gpu_launches": int(sum(c for _, c in stages.values())),
         "roofline": roof,
         "cpu_baseline": {"value": 1.0 / sec_per_pos, "unit": UNIT, "cores": blas_threads(), "kind": "oracle",

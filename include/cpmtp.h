@@ -53,7 +53,7 @@ enum {
   CPMTP_ERR_LIMIT = -7      /* size beyond a fixed built-in capacity */
 };
 
-enum { CPMTP_OP_FORWARD = 0, CPMTP_OP_BACKWARD = 1, CPMTP_OP_SCORE = 2 };
+enum { CPMTP_OP_FORWARD = 0, CPMTP_OP_BACKWARD = 1, CPMTP_OP_SCORE = 2, CPMTP_OP_SAMPLE = 3 };
 
 /* flags */
 #define CPMTP_FLAG_AUX 1u /* add aux_coef * sum_a wbar_a^2 to the loss (soft form of Eq. 10) */
@@ -134,6 +134,31 @@ int cpmtp_score_draft(const cpmtp_shape* shape, const void* h, const void* W_hea
                       cpmtp_stream stream);
 
 /*
+ * Generate a draft of n tokens per position from the factors (sampling section).
+ * Token s is drawn from  sum_a b_a P^(s)(v | a) / sum_a b_a  with
+ * b_a = w_a * prod_{t<s} P^(t)(x_t | a): Eq. 11 for the first token, and for the
+ * later ones the expert weights updated with the factors of the tokens already
+ * drawn, as the text under Eq. 12 describes (the printed Eq. 12 / Eq. 13 lack the
+ * s-th factor and the normaliser).  E and W_head are streamed once; the logits of
+ * the N*n*r rows are kept in the workspace (fp32) for the n sequential steps, so
+ * this entry point is meant for decode-sized N.
+ *   uniform [N,n,V] fp32, every value strictly inside (0,1), or NULL.  NULL: the
+ *     most likely token is taken (temperature 0; ties go to the lowest id).
+ *     Otherwise the token is argmax_v( log p(v) / temperature - log(-log uniform[v]) ),
+ *     an exact draw from the conditional sharpened by 1/temperature (> 0).
+ *   topk in [1, 8]: how many most-likely tokens of every conditional to report.
+ *   draft [N,n] int32 out.  logp_joint [N] fp32 out or NULL: Eq. 9 at the draft.
+ *   topk_tokens [N,n,topk] int32 / topk_logp [N,n,topk] fp32 out or NULL: the
+ *     candidates, best first, with their conditional log-probabilities (for a
+ *     static draft tree as in the speculative-decoding section).
+ */
+int cpmtp_sample_draft(const cpmtp_shape* shape, const void* h, const void* W_head, const void* E,
+                       const void* W_g, const float* uniform, float temperature, int32_t topk,
+                       int32_t* draft, float* logp_joint, int32_t* topk_tokens, float* topk_logp,
+                       void* workspace, size_t workspace_bytes, int32_t* dev_status,
+                       cpmtp_stream stream);
+
+/*
  * cpmtp_score_draft for callers that cannot hand over scratch memory.  Code that
  * runs where device allocation is off-limits -- inside a serving loop that has
  * frozen its memory pool, in a plugin that is given tensors but no allocator, or
@@ -202,6 +227,7 @@ enum {
   CPMTP_STAGE_DW_HEAD,
   CPMTP_STAGE_DH,
   CPMTP_STAGE_DW_G,
+  CPMTP_STAGE_DRAFT_STEP,    /* per-token selection passes of cpmtp_sample_draft */
   CPMTP_STAGE_COUNT
 };
 int cpmtp_profile_begin(void);

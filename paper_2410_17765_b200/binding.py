@@ -15,19 +15,19 @@ import torch
 
 from .build import LIB_PATH
 
-OP_FORWARD, OP_BACKWARD, OP_SCORE = 0, 1, 2
+OP_FORWARD, OP_BACKWARD, OP_SCORE, OP_SAMPLE = 0, 1, 2, 3
 FLAG_AUX = 1
 
 EXPORTS = [
     "cpmtp_version", "cpmtp_status_string", "cpmtp_workspace_bytes", "cpmtp_forward", "cpmtp_backward",
     "cpmtp_score_draft", "cpmtp_host_staging_bytes", "cpmtp_forward_host", "cpmtp_profile_begin",
-    "cpmtp_profile_end", "cpmtp_score_draft_static",
+    "cpmtp_profile_end", "cpmtp_score_draft_static", "cpmtp_sample_draft",
 ]
 
 STATIC_SCRATCH_BYTES = 4 << 20
 
 STAGES = ["gate", "proj", "lse", "mixture", "finalize", "coeff", "logit_grad", "dz", "de", "de_convert",
-          "dw_head", "dh", "dw_g"]
+          "dw_head", "dh", "dw_g", "draft_step"]
 
 
 class CShape(ctypes.Structure):
@@ -69,6 +69,9 @@ def load_library() -> ctypes.CDLL:
     lib.cpmtp_score_draft.argtypes = [shp, vp, vp, vp, vp, i32p, fp, fp, vp, sz, i32p, vp]
     lib.cpmtp_forward_host.restype = ctypes.c_int
     lib.cpmtp_forward_host.argtypes = [shp, vp, vp, vp, vp, i32p, fp, fp, svp, vp, sz, i32p, vp]
+    lib.cpmtp_sample_draft.restype = ctypes.c_int
+    lib.cpmtp_sample_draft.argtypes = [shp, vp, vp, vp, vp, fp, ctypes.c_float, ctypes.c_int32, i32p, fp, i32p, fp,
+                                       vp, sz, i32p, vp]
     lib.cpmtp_score_draft_static.restype = ctypes.c_int
     lib.cpmtp_score_draft_static.argtypes = [shp, vp, vp, vp, vp, i32p, fp, fp, i32p, vp]
     lib.cpmtp_profile_begin.restype = ctypes.c_int
@@ -226,6 +229,36 @@ def score_draft(h, W_head, E, W_g, draft, *, want_prefix: bool = True,
     rc = lib.cpmtp_score_draft(ctypes.byref(shape), _ptr(h), _ptr(W_head), _ptr(E), _ptr(W_g), _ptr(draft),
                                _ptr(res["logp_joint"]), _ptr(res.get("logp_prefix")) if want_prefix else None,
                                _ptr(workspace), workspace.numel(), _ptr(dev_status), _stream())
+    _check(rc)
+    return res
+
+
+def sample_draft(h, W_head, E, W_g, n: int, *, uniform: Optional[torch.Tensor] = None, temperature: float = 1.0,
+                 topk: int = 1, workspace: Optional[torch.Tensor] = None,
+                 dev_status: Optional[torch.Tensor] = None, out: Optional[dict] = None) -> dict:
+    """cpmtp_sample_draft; returns {"draft", "logp_joint", "topk_tokens", "topk_logp"} (device tensors).
+    uniform: [N, n, V] fp32 strictly inside (0, 1) for Gumbel-max sampling, or None for the greedy draft."""
+    lib = load_library()
+    N, d = h.shape
+    V, r = E.shape[0], W_g.shape[0]
+    assert W_head.shape == (n * r, d, d)
+    for t in (h, W_head, E, W_g):
+        assert t.dtype == torch.bfloat16 and t.is_contiguous()
+    if uniform is not None:
+        assert uniform.shape == (N, n, V) and uniform.dtype == torch.float32 and uniform.is_contiguous()
+    shape = make_shape(N, d, V, n, r)
+    if workspace is None:
+        workspace = alloc_workspace(workspace_bytes(shape, OP_SAMPLE), h.device)
+    res = out if out is not None else {}
+    dev = h.device
+    res.setdefault("draft", torch.empty((N, n), dtype=torch.int32, device=dev))
+    res.setdefault("logp_joint", torch.empty(N, dtype=torch.float32, device=dev))
+    res.setdefault("topk_tokens", torch.empty((N, n, topk), dtype=torch.int32, device=dev))
+    res.setdefault("topk_logp", torch.empty((N, n, topk), dtype=torch.float32, device=dev))
+    rc = lib.cpmtp_sample_draft(ctypes.byref(shape), _ptr(h), _ptr(W_head), _ptr(E), _ptr(W_g), _ptr(uniform),
+                                ctypes.c_float(temperature), topk, _ptr(res["draft"]), _ptr(res["logp_joint"]),
+                                _ptr(res["topk_tokens"]), _ptr(res["topk_logp"]), _ptr(workspace), workspace.numel(),
+                                _ptr(dev_status), _stream())
     _check(rc)
     return res
 

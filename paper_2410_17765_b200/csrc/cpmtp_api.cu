@@ -9,6 +9,7 @@
 #include <vector>
 
 #include "epilogues.cuh"
+#include "sampler_kernels.cuh"
 #include "small_kernels.cuh"
 #include "tc_gemm.cuh"
 #include "tmap.cuh"
@@ -206,6 +207,29 @@ struct ProfScope {
   }
 };
 
+struct SampleLayout {
+  FwdLayout fwd;
+  size_t logits, z32, lb, part_top, part_best, logp_tmp, total;
+  int lds, chunks;
+};
+
+SampleLayout sample_layout(const cpmtp_shape& s, int sms) {
+  SampleLayout L;
+  L.fwd = fwd_layout(s, sms);
+  L.lds = (s.V + 31) / 32 * 32;
+  L.chunks = (s.V + kSampleChunk - 1) / kSampleChunk;
+  size_t off = align_up(L.fwd.total);
+  auto take = [&](size_t bytes) { size_t o = off; off = align_up(off + bytes); return o; };
+  L.logits = take(sizeof(float) * static_cast<size_t>(L.fwd.M) * L.lds);
+  L.z32 = take(sizeof(float) * static_cast<size_t>(L.fwd.M) * s.d);
+  L.lb = take(sizeof(float) * s.N * s.r);
+  L.part_top = take(sizeof(Cand) * static_cast<size_t>(s.N) * L.chunks * kMaxTopk);
+  L.part_best = take(sizeof(Cand) * static_cast<size_t>(s.N) * L.chunks);
+  L.logp_tmp = take(sizeof(float) * s.N);
+  L.total = off;
+  return L;
+}
+
 template <class Cfg, class Epi>
 cudaError_t launch_gemm(const void* A, uint64_t a_rows, uint64_t a_ld, const void* B, uint64_t b_rows,
                         uint64_t b_ld, uint64_t kdim, const Sched& sched, const typename Epi::Params& ep,
@@ -256,7 +280,7 @@ cudaError_t gemm_auto(const void* A, uint64_t a_ld, const void* B, uint64_t b_ld
 int run_forward(const cpmtp_shape& s, const uint16_t* h, const uint16_t* W_head, const uint16_t* E,
                 const uint16_t* W_g, const int32_t* x, float* logp, float* loss, const cpmtp_saved* saved,
                 int32_t* counts, float* logp_prefix, uint8_t* ws, const FwdLayout& L, int* dev_status, int sms,
-                cudaStream_t stream) {
+                cudaStream_t stream, float* logits = nullptr, int lds = 0, float* z32 = nullptr) {
   float* logw = saved ? saved->logw : reinterpret_cast<float*>(ws + L.logw);
   float* q = saved ? saved->q : reinterpret_cast<float*>(ws + L.q);
   float* wbar = saved ? saved->wbar : reinterpret_cast<float*>(ws + L.wbar);
@@ -272,7 +296,7 @@ int run_forward(const cpmtp_shape& s, const uint16_t* h, const uint16_t* W_head,
   // head projection: z[N, K*d] = h[N, d] * W_cat[K*d, d]^T, plus the fp32 target-logit partials
   {
     ProfScope prof(CPMTP_STAGE_PROJ, stream);
-    EpiProj<kBN>::Params ep{z, tgt_part, E, x, dev_status, s.N, ncols, s.d, s.V, s.n, s.r};
+    EpiProj<kBN>::Params ep{z, tgt_part, E, x, z32, dev_status, s.N, ncols, s.d, s.V, s.n, s.r};
     if (s.N <= CfgKKSkinny::A_ROWS) {
       const int n_tiles = (ncols + kBN - 1) / kBN;
       const Sched sc = make_sched(1, n_tiles, n_tiles, 1, s.d / kBK);
@@ -284,13 +308,24 @@ int run_forward(const cpmtp_shape& s, const uint16_t* h, const uint16_t* W_head,
   // unembedding fused with the vocabulary log-sum-exp (Eq. 6, Eq. 8)
   {
     ProfScope prof(CPMTP_STAGE_LSE, stream);
-    EpiLse<kBN>::Params ep{part_m, part_l, L.M, s.V, L.lse_sched.n_splits};
-    if (L.M <= CfgKKSkinny::A_ROWS) {
-      CPMTP_TRY((launch_gemm<CfgKKSkinny, EpiLse<kBN>>(z, L.M, s.d, E, s.V, s.d, s.d, L.lse_sched, ep, dev_status, sms, stream)));
-    } else if (L.wide) {
-      CPMTP_TRY((launch_gemm<WideKK, EpiLse<kBN>>(z, L.M, s.d, E, s.V, s.d, s.d, L.lse_sched, ep, dev_status, sms, stream)));
+    if (logits != nullptr) {
+      EpiLse<kBN, true>::Params ep{part_m, part_l, L.M, s.V, L.lse_sched.n_splits, logits, lds};
+      if (L.M <= CfgKKSkinny::A_ROWS) {
+        CPMTP_TRY((launch_gemm<CfgKKSkinny, EpiLse<kBN, true>>(z, L.M, s.d, E, s.V, s.d, s.d, L.lse_sched, ep, dev_status, sms, stream)));
+      } else if (L.wide) {
+        CPMTP_TRY((launch_gemm<WideKK, EpiLse<kBN, true>>(z, L.M, s.d, E, s.V, s.d, s.d, L.lse_sched, ep, dev_status, sms, stream)));
+      } else {
+        CPMTP_TRY((launch_gemm<CfgKK, EpiLse<kBN, true>>(z, L.M, s.d, E, s.V, s.d, s.d, L.lse_sched, ep, dev_status, sms, stream)));
+      }
     } else {
-      CPMTP_TRY((launch_gemm<CfgKK, EpiLse<kBN>>(z, L.M, s.d, E, s.V, s.d, s.d, L.lse_sched, ep, dev_status, sms, stream)));
+      EpiLse<kBN>::Params ep{part_m, part_l, L.M, s.V, L.lse_sched.n_splits, nullptr, 0};
+      if (L.M <= CfgKKSkinny::A_ROWS) {
+        CPMTP_TRY((launch_gemm<CfgKKSkinny, EpiLse<kBN>>(z, L.M, s.d, E, s.V, s.d, s.d, L.lse_sched, ep, dev_status, sms, stream)));
+      } else if (L.wide) {
+        CPMTP_TRY((launch_gemm<WideKK, EpiLse<kBN>>(z, L.M, s.d, E, s.V, s.d, s.d, L.lse_sched, ep, dev_status, sms, stream)));
+      } else {
+        CPMTP_TRY((launch_gemm<CfgKK, EpiLse<kBN>>(z, L.M, s.d, E, s.V, s.d, s.d, L.lse_sched, ep, dev_status, sms, stream)));
+      }
     }
   }
   // gate (Eq. 7) and mixture epilogue (Eq. 9)
@@ -298,7 +333,8 @@ int run_forward(const cpmtp_shape& s, const uint16_t* h, const uint16_t* W_head,
     ProfScope prof(CPMTP_STAGE_MIXTURE, stream);
     const int threads = s.N <= 256 ? 1024 : 256;
     gate_mixture_kernel<<<s.N, threads, 0, stream>>>(h, W_g, s.d, part_m, part_l, L.lse_sched.n_splits, tgt_part,
-                                                    s.d / 64, logw, lse, tgt, q, logp, logp_prefix, s.N, s.n, s.r);
+                                                    x != nullptr ? s.d / 64 : 0, logw, lse, tgt, q, logp, logp_prefix,
+                                                    s.N, s.n, s.r);
     CPMTP_TRY(cudaGetLastError());
   }
   if (loss != nullptr || counts != nullptr || saved != nullptr) {
@@ -418,6 +454,7 @@ size_t cpmtp_workspace_bytes(const cpmtp_shape* shape, int op) {
     case CPMTP_OP_FORWARD:
     case CPMTP_OP_SCORE: return fwd_layout(*shape, sms).total;
     case CPMTP_OP_BACKWARD: return bwd_layout(*shape).total;
+    case CPMTP_OP_SAMPLE: return sample_layout(*shape, sms).total;
     default: return 0;
   }
 }
@@ -460,6 +497,50 @@ int cpmtp_score_draft(const cpmtp_shape* shape, const void* h, const void* W_hea
                      static_cast<const uint16_t*>(E), static_cast<const uint16_t*>(W_g), draft, logp_joint,
                      nullptr, nullptr, nullptr, logp_prefix, static_cast<uint8_t*>(workspace), L, dev_status,
                      di->sms, reinterpret_cast<cudaStream_t>(stream));
+}
+
+int cpmtp_sample_draft(const cpmtp_shape* shape, const void* h, const void* W_head, const void* E,
+                       const void* W_g, const float* uniform, float temperature, int32_t topk, int32_t* draft,
+                       float* logp_joint, int32_t* topk_tokens, float* topk_logp, void* workspace,
+                       size_t workspace_bytes, int32_t* dev_status, cpmtp_stream stream) {
+  DeviceInfo* di = nullptr;
+  const int rc = check_common(shape, h, W_head, E, W_g, /*x=*/h, workspace, &di);
+  if (rc != CPMTP_OK) return rc;
+  if (draft == nullptr) return CPMTP_ERR_NULL;
+  if (topk < 1 || topk > kMaxTopk || topk > shape->V) return CPMTP_ERR_SHAPE;
+  if (uniform != nullptr && !(temperature > 0.f)) return CPMTP_ERR_SHAPE;
+  const cpmtp_shape& s = *shape;
+  const SampleLayout L = sample_layout(s, di->sms);
+  if (workspace_bytes < L.total) return CPMTP_ERR_WORKSPACE;
+  cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
+  uint8_t* ws = static_cast<uint8_t*>(workspace);
+  float* logits = reinterpret_cast<float*>(ws + L.logits);
+  float* lb = reinterpret_cast<float*>(ws + L.lb);
+  float* z32 = reinterpret_cast<float*>(ws + L.z32);
+  Cand* part_top = reinterpret_cast<Cand*>(ws + L.part_top);
+  Cand* part_best = reinterpret_cast<Cand*>(ws + L.part_best);
+  float* logp_tmp = reinterpret_cast<float*>(ws + L.logp_tmp);
+  float* logw = reinterpret_cast<float*>(ws + L.fwd.logw);
+  float* lse = reinterpret_cast<float*>(ws + L.fwd.lse);
+  // projection, unembedding (logits kept) and gate: the forward pipeline without targets
+  const int rf = run_forward(s, static_cast<const uint16_t*>(h), static_cast<const uint16_t*>(W_head),
+                             static_cast<const uint16_t*>(E), static_cast<const uint16_t*>(W_g), nullptr, logp_tmp,
+                             nullptr, nullptr, nullptr, nullptr, ws, L.fwd, dev_status, di->sms, st, logits, L.lds, z32);
+  if (rf != CPMTP_OK) return rf;
+  CPMTP_TRY(cudaMemcpyAsync(lb, logw, sizeof(float) * s.N * s.r, cudaMemcpyDeviceToDevice, st));   // b = w
+  const float inv_temp = uniform != nullptr ? 1.0f / temperature : 1.0f;
+  for (int step = 0; step < s.n; ++step) {
+    ProfScope prof(CPMTP_STAGE_DRAFT_STEP, st);
+    draft_step_partial_kernel<<<dim3(L.chunks, s.N), kSampleThreads, 0, st>>>(
+        logits, L.lds, lse, lb, uniform, inv_temp, step, s.V, s.n, s.r, topk, part_top, part_best);
+    CPMTP_TRY(cudaGetLastError());
+    draft_step_final_kernel<<<s.N, kSampleThreads, 0, st>>>(z32, static_cast<const uint16_t*>(E), s.d, lse, lb,
+                                                           part_top, part_best, L.chunks,
+                                                           uniform != nullptr ? 1 : 0, step, s.V, s.n, s.r, topk,
+                                                           draft, logp_joint, topk_tokens, topk_logp);
+    CPMTP_TRY(cudaGetLastError());
+  }
+  return CPMTP_OK;
 }
 
 int cpmtp_score_draft_static(const cpmtp_shape* shape, const void* h, const void* W_head, const void* E,

@@ -62,7 +62,8 @@ struct EpiProj {
     uint16_t* z;            // [M, ncols] bf16
     float* tgt_part;        // [M, ncols / 64]
     const uint16_t* E;      // [V, d] bf16
-    const int32_t* x;       // [M, n]
+    const int32_t* x;       // [M, n], or nullptr to skip the target-logit side output
+    float* z32;             // [M, ncols] unrounded z for the draft sampler, or nullptr
     int* dev_status;
     int M, ncols, d, V, n, r;
   };
@@ -84,6 +85,13 @@ struct EpiProj {
       ptx::tmem_ld_32x32(tacc + c, v);
       ptx::tmem_ld_wait();
       if (valid) {
+        store_bf16x32(p.z + static_cast<size_t>(row) * p.ncols + col0, v);
+        if (p.z32 != nullptr) {
+          float4* dst = reinterpret_cast<float4*>(p.z32 + static_cast<size_t>(row) * p.ncols + col0);
+#pragma unroll
+          for (int q = 0; q < 8; ++q) dst[q] = make_float4(v[q * 4], v[q * 4 + 1], v[q * 4 + 2], v[q * 4 + 3]);
+        }
+        if (p.x == nullptr) continue;   // no targets (draft generation): only z is needed
         const int k = col0 / p.d;
         const int j0 = col0 - k * p.d;
         int tok = p.x[static_cast<size_t>(row) * p.n + k / p.r];
@@ -95,7 +103,6 @@ struct EpiProj {
         float acc = 0.f;
 #pragma unroll
         for (int q = 0; q < 4; ++q) acc = dot8(__ldg(e + q), v + q * 8, acc);
-        store_bf16x32(p.z + static_cast<size_t>(row) * p.ncols + col0, v);
         if ((c & 32) == 0) {
           part = acc;
         } else {
@@ -111,12 +118,16 @@ struct EpiProj {
 //   S[(i,k), v] = E[v, :] . z[i, k, :] never leaves TMEM/registers; each thread
 // keeps a running (max, sum-exp) over the column tiles of its unit and writes
 // one partial per (row, split).  Values are kept in the log2 domain.
-template <int BN>
+// STORE = true additionally writes the raw logits (fp32) for the draft sampler, which needs
+// whole distributions; the likelihood path never does.
+template <int BN, bool STORE = false>
 struct EpiLse {
   struct Params {
     float* part_m;   // [M, splits] running max * log2(e)
     float* part_l;   // [M, splits] sum 2^(s*log2e - max)
     int M, V, splits;
+    float* S;        // [M, lds] logits (STORE only); lds % 32 == 0, lds >= V
+    int lds;
   };
   struct State { float m2, l; };
   static constexpr int SMEM_BYTES = 0;
@@ -132,8 +143,8 @@ struct EpiLse {
       p.part_l[static_cast<size_t>(row) * p.splits + split] = st.l;
     }
   }
-  __device__ static void tile(const Params& p, State& st, uint32_t tacc, int, int n_tile, int, uint8_t*,
-                              int) {
+  __device__ static void tile(const Params& p, State& st, uint32_t tacc, int m_tile, int n_tile,
+                              int row_in_tile, uint8_t*, int) {
 #pragma unroll 1
     for (int c = 0; c < BN; c += 32) {
       const int col0 = n_tile * BN + c;
@@ -141,6 +152,14 @@ struct EpiLse {
       float v[32];
       ptx::tmem_ld_32x32(tacc + c, v);
       ptx::tmem_ld_wait();
+      if constexpr (STORE) {
+        const int row = m_tile * kBM + row_in_tile;
+        if (row < p.M) {
+          float4* dst = reinterpret_cast<float4*>(p.S + static_cast<size_t>(row) * p.lds + col0);
+#pragma unroll
+          for (int q = 0; q < 8; ++q) dst[q] = make_float4(v[q * 4], v[q * 4 + 1], v[q * 4 + 2], v[q * 4 + 3]);
+        }
+      }
       if (col0 + 32 > p.V) {
 #pragma unroll
         for (int j = 0; j < 32; ++j)

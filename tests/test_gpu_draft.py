@@ -1,0 +1,109 @@
+"""GPU parity of draft generation (cpmtp_sample_draft) against the fp64 oracle.
+
+A drafted token is an argmax, so a near-tie may legitimately resolve differently in
+fp32: tokens are compared exactly where the oracle's margin is clear, and otherwise
+the GPU's choice must be within the tolerance of the oracle's best score.  What is
+unique is compared outright: the joint log-probability of the GPU's own draft (the
+oracle's likelihood of those tokens) and the candidates' conditional log-probabilities."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import cp_head
+from paper_2410_17765_b200 import synth
+
+pytestmark = pytest.mark.gpu
+
+LOGP_TOL = 2e-3
+
+
+def to_dev(inp):
+    return [t.cuda() for t in (inp.h, inp.W_head, inp.E, inp.W_g)]
+
+
+def check_against_oracle(inp, out, ref, topk, uniform=None, temperature=1.0):
+    s = inp.shape
+    draft = out["draft"].cpu().numpy().astype(np.int64)
+    assert draft.min() >= 0 and draft.max() < s.V
+    # 1. joint log-probability of the GPU's own draft
+    fw = cp_head.forward(inp.h, inp.W_head, inp.E, inp.W_g, torch.from_numpy(draft), s.n, s.r)
+    assert np.max(np.abs(out["logp_joint"].cpu().numpy() - fw.logp)) <= LOGP_TOL
+    # 2. tokens: follow the oracle position by position while the prefixes agree
+    tk = out["topk_tokens"].cpu().numpy()
+    tl = out["topk_logp"].cpu().numpy()
+    same_prefix = np.ones(s.N, dtype=bool)
+    agree = 0
+    for t in range(s.n):
+        mix = ref.mix[:, t, :]
+        norm = cp_head.logsumexp(mix, axis=1) if t == 0 else None
+        for i in np.nonzero(same_prefix)[0]:
+            if uniform is None:
+                score = mix[i]
+            else:
+                cond = mix[i] - cp_head.logsumexp(ref.mix[i, t][None, :], axis=1)[0]
+                score = cond / temperature - np.log(-np.log(uniform[i, t].double().numpy()))
+            best = score.max()
+            assert score[draft[i, t]] >= best - 2 * LOGP_TOL / min(1.0, temperature), (i, t)
+            if draft[i, t] == ref.tokens[i, t]:
+                agree += 1
+                # candidates of this conditional: same scores (the order of near-equal ones may differ)
+                want = ref.topk_logp[i, t]
+                assert np.max(np.abs(np.sort(tl[i, t])[::-1] - want)) <= 3 * LOGP_TOL, (i, t)
+                cond_all = mix[i] - cp_head.logsumexp(mix[i][None, :], axis=1)[0]
+                assert np.max(np.abs(cond_all[tk[i, t]] - tl[i, t])) <= LOGP_TOL
+                assert len(set(tk[i, t].tolist())) == topk
+            else:
+                same_prefix[i] = False
+    return agree / (s.N * s.n)
+
+
+@pytest.mark.parametrize("N,V,d,n,r,topk", [(8, 5000, 256, 4, 8, 5), (1, 3000, 512, 3, 4, 1), (64, 2500, 128, 2, 3, 8),
+                                            (5, 130, 64, 8, 32, 2)])
+def test_greedy_draft_matches_oracle(N, V, d, n, r, topk):
+    from paper_2410_17765_b200 import binding
+
+    shape = synth.Shape(N=N, d=d, V=V, n=n, r=r)
+    inp = synth.make_inputs(shape, seed=7, weight_scale=2.0)
+    ref = cp_head.draft(inp.h, inp.W_head, inp.E, inp.W_g, n, r, topk=topk)
+    st = torch.zeros(1, dtype=torch.int32, device="cuda")
+    out = binding.sample_draft(*to_dev(inp), n, topk=topk, dev_status=st)
+    torch.cuda.synchronize()
+    assert int(st.item()) == 0
+    frac = check_against_oracle(inp, out, ref, topk)
+    assert frac >= 0.9
+    # greedy: the first candidate is the drafted token
+    assert torch.equal(out["topk_tokens"][:, :, 0], out["draft"])
+
+
+def test_sampled_draft_matches_oracle():
+    from paper_2410_17765_b200 import binding
+
+    shape = synth.Shape(N=16, d=256, V=4000, n=3, r=4)
+    inp = synth.make_inputs(shape, seed=9, weight_scale=2.0)
+    g = torch.Generator().manual_seed(5)
+    u = torch.rand((shape.N, shape.n, shape.V), generator=g, dtype=torch.float32).clamp_(1e-7, 1 - 1e-7)
+    for temperature in (1.0, 0.5):
+        ref = cp_head.draft(inp.h, inp.W_head, inp.E, inp.W_g, shape.n, shape.r, topk=4, uniform=u,
+                            temperature=temperature)
+        out = binding.sample_draft(*to_dev(inp), shape.n, uniform=u.cuda(), temperature=temperature, topk=4)
+        torch.cuda.synchronize()
+        frac = check_against_oracle(inp, out, ref, 4, uniform=u, temperature=temperature)
+        assert frac >= 0.9
+    # sampling spreads over tokens: not every position takes the most likely one
+    assert not torch.equal(out["topk_tokens"][:, :, 0], out["draft"])
+
+
+def test_draft_is_deterministic_and_validates_arguments():
+    from paper_2410_17765_b200 import binding
+
+    shape = synth.Shape(N=4, d=128, V=900, n=2, r=2)
+    inp = synth.make_inputs(shape, seed=2)
+    dev = to_dev(inp)
+    a = binding.sample_draft(*dev, shape.n, topk=3)
+    b = binding.sample_draft(*dev, shape.n, topk=3)
+    torch.cuda.synchronize()
+    assert torch.equal(a["draft"], b["draft"]) and torch.equal(a["topk_logp"], b["topk_logp"])
+    with pytest.raises(binding.CpmtpError):
+        binding.sample_draft(*dev, shape.n, topk=9)
+    with pytest.raises(binding.CpmtpError):
+        binding.sample_draft(*dev, shape.n, uniform=torch.rand((4, 2, 900), device="cuda"), temperature=0.0)

@@ -142,6 +142,39 @@ def test_decode_full_size(name, count):
     assert np.max(np.abs(out["logp_prefix"].cpu().numpy()[idx.numpy()] - pre)) <= LOGP_TOL
 
 
+def test_draft_generation_full_decode_size():
+    """Greedy draft with 5 candidates at the decode shape (N=8, d=4096, V=128256, n=4, r=8)."""
+    from paper_2410_17765_b200 import binding
+
+    inp = inputs_for("decode_8")
+    s = inp.shape
+    ref = cp_head.draft(inp.h, inp.W_head, inp.E, inp.W_g, s.n, s.r, topk=5)
+    st = torch.zeros(1, dtype=torch.int32, device="cuda")
+    h, W, E, Wg, _ = to_dev(inp)
+    out = binding.sample_draft(h, W, E, Wg, s.n, topk=5, dev_status=st)
+    torch.cuda.synchronize()
+    assert int(st.item()) == 0
+    draft = out["draft"].cpu().numpy().astype(np.int64)
+    fw = cp_head.forward(inp.h, inp.W_head, inp.E, inp.W_g, torch.from_numpy(draft), s.n, s.r)
+    assert np.max(np.abs(out["logp_joint"].cpu().numpy() - fw.logp)) <= LOGP_TOL
+    tl = out["topk_logp"].cpu().numpy()
+    agree = 0
+    for i in range(s.N):
+        for t in range(s.n):
+            # the drafted token is the oracle's argmax or within tolerance of it
+            assert ref.mix[i, t, draft[i, t]] >= ref.mix[i, t].max() - 5 * LOGP_TOL
+            if draft[i, t] != ref.tokens[i, t]:
+                break
+            agree += 1
+            # candidate values are exact (unrounded z); the candidate *set* is selected on bf16-z logits,
+            # so the last place may go to a token within the selection's resolution of the true k-th
+            assert np.max(np.abs(np.sort(tl[i, t])[::-1] - ref.topk_logp[i, t])) <= 5 * LOGP_TOL
+            cond = ref.mix[i, t] - cp_head.logsumexp(ref.mix[i, t][None, :], axis=1)[0]
+            tk = out["topk_tokens"][i, t].cpu().numpy()
+            assert np.max(np.abs(cond[tk] - tl[i, t])) <= LOGP_TOL
+    assert agree >= 0.75 * s.N * s.n
+
+
 def test_bigvocab_full_size_forward_and_backward_sampled():
     from paper_2410_17765_b200 import binding
 
