@@ -258,3 +258,73 @@ def draft(h, W_head, E, W_g, n: int, r: int, *, topk: int = 1, uniform=None,
         lb = lb + logP[rows, s, :, x_s]
     return Draft(tokens=tokens, logp_joint=logsumexp(lb, axis=1), topk_tokens=top_t, topk_logp=top_lp,
                  mix=mixes)
+
+
+# ---------------------------------------------------------------------------
+# Full head (Eq. 6 as printed): one unembedding W^(s)_alpha in R^{V x d} per (token, expert),
+# stacked as W_full[k, V, d] with k = s*r + alpha.  The shared-head form above is the special
+# case W_full[k] = E . W_head[k].
+
+
+def factor_log_probs_full(h, W_full, x, n: int, r: int):
+    """C, lse, tgt as in factor_log_probs, with logits S[i, k, :] = W_full[k] . h[i] (Eq. 6, Eq. 8)."""
+    hd, xi = _f64(h), _i64(x)
+    N = hd.shape[0]
+    K = n * r
+    lse = np.empty((N, K))
+    tgt = np.empty((N, K))
+    rows = np.arange(N)
+    for k in range(K):
+        S = hd @ _f64(W_full[k]).T
+        lse[:, k] = logsumexp(S, axis=1)
+        tgt[:, k] = S[rows, xi[:, k // r]]
+    return (tgt - lse).reshape(N, n, r), lse, tgt
+
+
+def forward_full(h, W_full, W_g, x, n: int, r: int, *, aux_coef: float = 0.0) -> Forward:
+    """Eq. 9 with the full head of Eq. 6."""
+    logw = gate_log_weights(h, W_g)
+    C, lse, tgt = factor_log_probs_full(h, W_full, x, n, r)
+    a = logw + C.sum(axis=1)
+    logp = logsumexp(a, axis=1)
+    q = np.exp(a - logp[:, None])
+    w = np.exp(logw)
+    wbar = w.mean(axis=0)
+    counts = np.bincount(np.argmax(w, axis=1), minlength=r).astype(np.int64)
+    loss = float(-logp.mean() + aux_coef * np.sum(wbar * wbar))
+    return Forward(logp=logp, logw=logw, C=C, lse=lse, tgt=tgt, a=a, q=q, wbar=wbar, counts=counts, loss=loss)
+
+
+@dataclass
+class GradientsFull:
+    dh: np.ndarray       # [N, d]
+    dW_full: np.ndarray  # [n*r, V, d]
+    dW_g: np.ndarray     # [r, d]
+
+
+def backward_full(h, W_full, W_g, x, n: int, r: int, *, aux_coef: float = 0.0, dloss_dlogp=None) -> GradientsFull:
+    """Gradient of the same objective as `backward`, for the full head:
+    dS as there; dW_full[k] = dS[:, k, :]^T h, dh = sum_k dS[:, k, :] W_full[k] + dg W_g."""
+    hd, Wg, xi = _f64(h), _f64(W_g), _i64(x)
+    N, d = hd.shape
+    K = n * r
+    fw = forward_full(h, W_full, W_g, x, n, r, aux_coef=aux_coef)
+    up = np.full(N, -1.0 / N) if dloss_dlogp is None else _f64(dloss_dlogp)
+    c = up[:, None] * fw.q
+    w = np.exp(fw.logw)
+    u = 2.0 * aux_coef * fw.wbar / N
+    dg = up[:, None] * (fw.q - w) + w * (u[None, :] - (w @ u)[:, None])
+    dh = dg @ Wg
+    dW_g = dg.T @ hd
+    V = _f64(W_full[0]).shape[0]
+    dW_full = np.empty((K, V, d))
+    rows = np.arange(N)
+    for k in range(K):
+        s, alpha = divmod(k, r)
+        Wk = _f64(W_full[k])
+        S = hd @ Wk.T
+        G = -c[:, alpha][:, None] * np.exp(S - fw.lse[:, k][:, None])
+        G[rows, xi[:, s]] += c[:, alpha]
+        dW_full[k] = G.T @ hd
+        dh += G @ Wk
+    return GradientsFull(dh=dh, dW_full=dW_full, dW_g=dW_g)
