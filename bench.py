@@ -35,6 +35,7 @@ WORKLOADS = {
     "decode_8": ("decode_8", "score", {}, None),
     "decode_64": ("decode_64", "score", {}, None),
     "draft_8": ("decode_8", "sample", {}, None),
+    "full_head_fwd_bwd": ("full_head_train", "full_fwd_bwd", {}, None),
     "train_fwd_bwd_small": ("train_fwd_bwd_small", "fwd_bwd", {}, None),
     "bigvocab_fwd_small": ("bigvocab_fwd_small", "fwd", {"targets": "zipf"}, 1.0),
     "tiny": ("tiny", "fwd_bwd", {}, None),
@@ -102,6 +103,8 @@ class ClockSampler:
 def flops_per_position(s, kind):
     K = s.n * s.r
     fwd = 2 * K * (s.d * s.d + s.V * s.d) + 2 * s.r * s.d
+    if kind == "full_fwd_bwd":
+        return 3 * (2 * K * s.V * s.d + 2 * s.r * s.d)
     return fwd if kind != "fwd_bwd" else 3 * fwd
 
 
@@ -115,7 +118,9 @@ def oracle_seconds_per_position(inp, kind, aux, sample: int):
     sample = min(sample, s.N)
     sub = synth.subsample_positions(inp, torch.arange(sample))
     t0 = time.perf_counter()
-    if kind == "fwd_bwd":
+    if kind == "full_fwd_bwd":
+        cp_head.backward_full(sub.h, synth.make_full_head(s, seed=0), sub.W_g, sub.x, s.n, s.r, aux_coef=aux or 0.0)
+    elif kind == "fwd_bwd":
         cp_head.backward(sub.h, sub.W_head, sub.E, sub.W_g, sub.x, s.n, s.r, aux_coef=aux or 0.0)
     else:
         cp_head.forward(sub.h, sub.W_head, sub.E, sub.W_g, sub.x, s.n, s.r, aux_coef=aux or 0.0)
@@ -192,6 +197,12 @@ def run_ours(args, rank: int, world: int, local_rank: int):
                                      binding.host_staging_bytes(cs) + 512)
     status = torch.zeros(1, dtype=torch.int32, device="cuda")
     saved = binding.Saved.alloc(cs) if kind == "fwd_bwd" else None
+    W_full = ws_ff = ws_fb = None
+    if kind == "full_fwd_bwd":
+        W_full = synth.make_full_head(shape, seed=dist_util.shard_seed(0, rank)).cuda()
+        saved = binding.Saved.alloc_full(cs)
+        ws_ff = binding.alloc_workspace(binding.workspace_bytes(cs, binding.OP_FORWARD_FULL))
+        ws_fb = binding.alloc_workspace(binding.workspace_bytes(cs, binding.OP_BACKWARD_FULL))
     ws_bwd = binding.alloc_workspace(binding.workspace_bytes(cs, binding.OP_BACKWARD)) if kind == "fwd_bwd" else None
     ws_smp = binding.alloc_workspace(binding.workspace_bytes(cs, binding.OP_SAMPLE)) if kind == "sample" else None
     out_f, out_b, out_s = {}, {}, {}
@@ -206,6 +217,9 @@ def run_ours(args, rank: int, world: int, local_rank: int):
                              out=out_b)
         elif kind == "sample":
             binding.sample_draft(h, W_head, E, W_g, shape.n, topk=5, workspace=ws_smp, dev_status=status, out=out_s)
+        elif kind == "full_fwd_bwd":
+            binding.forward_full(h, W_full, W_g, x, saved=saved, workspace=ws_ff, dev_status=status, out=out_f)
+            binding.backward_full(h, W_full, W_g, x, saved, workspace=ws_fb, dev_status=status, out=out_b)
         else:
             binding.score_draft(h, W_head, E, W_g, x, workspace=ws_fwd, dev_status=status, out=out_s)
 
@@ -220,6 +234,13 @@ def run_ours(args, rank: int, world: int, local_rank: int):
             h.copy_(h_pin, non_blocking=True)
             binding.sample_draft(h, W_head, E, W_g, shape.n, topk=5, workspace=ws_smp, dev_status=status, out=out_s)
             draft_pin.copy_(out_s["draft"], non_blocking=True)
+            torch.cuda.current_stream().synchronize()
+            return
+        if kind == "full_fwd_bwd":
+            h.copy_(h_pin, non_blocking=True)
+            x.copy_(x_pin, non_blocking=True)
+            step()
+            loss_pin.copy_(out_f["loss"], non_blocking=True)
             torch.cuda.current_stream().synchronize()
             return
         binding.forward_host(h_pin, W_head, E, W_g, x_pin, logp_pin, loss_pin, aux_coef=aux, saved=saved,
@@ -283,6 +304,8 @@ def run_ours(args, rank: int, world: int, local_rank: int):
     roof["frac"] = roof["achieved"] / roof["peak"]
     roof["traffic"] = NCU_TRAFFIC_BYTES.get(args.workload)
     roof["kernel"] = "tc_gemm_kernel<EpiLse> (unembedding + logsumexp_V)"
+    if kind == "full_fwd_bwd":
+        roof["kernel"] = "tc_gemm_kernel<EpiLseFull> (all heads' unembeddings + logsumexp_V in one GEMM)"
     roof["peak_source"] = peaks["src"]
     roof["avg_launch_ms"] = avg_ms
     roof["algorithmic_per_launch"] = alg

@@ -53,7 +53,14 @@ enum {
   CPMTP_ERR_LIMIT = -7      /* size beyond a fixed built-in capacity */
 };
 
-enum { CPMTP_OP_FORWARD = 0, CPMTP_OP_BACKWARD = 1, CPMTP_OP_SCORE = 2, CPMTP_OP_SAMPLE = 3 };
+enum {
+  CPMTP_OP_FORWARD = 0,
+  CPMTP_OP_BACKWARD = 1,
+  CPMTP_OP_SCORE = 2,
+  CPMTP_OP_SAMPLE = 3,
+  CPMTP_OP_FORWARD_FULL = 4,
+  CPMTP_OP_BACKWARD_FULL = 5
+};
 
 /* flags */
 #define CPMTP_FLAG_AUX 1u /* add aux_coef * sum_a wbar_a^2 to the loss (soft form of Eq. 10) */
@@ -157,6 +164,31 @@ int cpmtp_sample_draft(const cpmtp_shape* shape, const void* h, const void* W_he
                        int32_t* draft, float* logp_joint, int32_t* topk_tokens, float* topk_logp,
                        void* workspace, size_t workspace_bytes, int32_t* dev_status,
                        cpmtp_stream stream);
+
+/*
+ * The same log-likelihood with the FULL head of Eq. 6 as printed: one unembedding
+ * W^(s)_a in R^{V x d} per (token, expert) instead of E . W_head[s, a],
+ *   S[i, s, a, :] = W_full[s*r + a] h[i],     W_full [n*r, V, d] bf16,
+ * the parametrisation used when the model is trained from scratch.  All n*r heads
+ * run as one GEMM over h; Eq. 8's vocabulary reduction is fused as above and the
+ * target logit is read from the fp32 accumulator.  Other arguments as for
+ * cpmtp_forward; `saved->z` is not used and may be NULL; logp_prefix [N,n] (or NULL)
+ * as for cpmtp_score_draft.  Workspace: CPMTP_OP_FORWARD_FULL.
+ */
+int cpmtp_forward_full(const cpmtp_shape* shape, const void* h, const void* W_full, const void* W_g,
+                       const int32_t* x, float* logp, float* loss, float* logp_prefix,
+                       const cpmtp_saved* saved, int32_t* expert_counts, void* workspace,
+                       size_t workspace_bytes, int32_t* dev_status, cpmtp_stream stream);
+
+/*
+ * Gradients for the full head (same objective and conventions as cpmtp_backward):
+ *   dh [N,d], dW_full [n*r,V,d], dW_g [r,d], bf16, all required.
+ * The logits are recomputed a few heads at a time.  Workspace: CPMTP_OP_BACKWARD_FULL.
+ */
+int cpmtp_backward_full(const cpmtp_shape* shape, const void* h, const void* W_full, const void* W_g,
+                        const int32_t* x, const cpmtp_saved* saved, const float* dloss_dlogp,
+                        void* dh, void* dW_full, void* dW_g, void* workspace,
+                        size_t workspace_bytes, int32_t* dev_status, cpmtp_stream stream);
 
 /*
  * cpmtp_score_draft for callers that cannot hand over scratch memory.  Code that

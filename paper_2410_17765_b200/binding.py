@@ -15,13 +15,14 @@ import torch
 
 from .build import LIB_PATH
 
-OP_FORWARD, OP_BACKWARD, OP_SCORE, OP_SAMPLE = 0, 1, 2, 3
+OP_FORWARD, OP_BACKWARD, OP_SCORE, OP_SAMPLE, OP_FORWARD_FULL, OP_BACKWARD_FULL = 0, 1, 2, 3, 4, 5
 FLAG_AUX = 1
 
 EXPORTS = [
     "cpmtp_version", "cpmtp_status_string", "cpmtp_workspace_bytes", "cpmtp_forward", "cpmtp_backward",
     "cpmtp_score_draft", "cpmtp_host_staging_bytes", "cpmtp_forward_host", "cpmtp_profile_begin",
     "cpmtp_profile_end", "cpmtp_score_draft_static", "cpmtp_sample_draft",
+    "cpmtp_forward_full", "cpmtp_backward_full",
 ]
 
 STATIC_SCRATCH_BYTES = 4 << 20
@@ -72,6 +73,10 @@ def load_library() -> ctypes.CDLL:
     lib.cpmtp_sample_draft.restype = ctypes.c_int
     lib.cpmtp_sample_draft.argtypes = [shp, vp, vp, vp, vp, fp, ctypes.c_float, ctypes.c_int32, i32p, fp, i32p, fp,
                                        vp, sz, i32p, vp]
+    lib.cpmtp_forward_full.restype = ctypes.c_int
+    lib.cpmtp_forward_full.argtypes = [shp, vp, vp, vp, i32p, fp, fp, fp, svp, i32p, vp, sz, i32p, vp]
+    lib.cpmtp_backward_full.restype = ctypes.c_int
+    lib.cpmtp_backward_full.argtypes = [shp, vp, vp, vp, i32p, svp, fp, vp, vp, vp, vp, sz, i32p, vp]
     lib.cpmtp_score_draft_static.restype = ctypes.c_int
     lib.cpmtp_score_draft_static.argtypes = [shp, vp, vp, vp, vp, i32p, fp, fp, i32p, vp]
     lib.cpmtp_profile_begin.restype = ctypes.c_int
@@ -139,6 +144,15 @@ class Saved:
     q: torch.Tensor
     wbar: torch.Tensor
     z: torch.Tensor
+
+    @staticmethod
+    def alloc_full(shape: CShape, device="cuda") -> "Saved":
+        """Saved state for the full-head entry points (no projected hidden states)."""
+        K = shape.n * shape.r
+        f = dict(dtype=torch.float32, device=device)
+        return Saved(lse=torch.empty((shape.N, K), **f), tgt=torch.empty((shape.N, K), **f),
+                     logw=torch.empty((shape.N, shape.r), **f), q=torch.empty((shape.N, shape.r), **f),
+                     wbar=torch.empty((32,), **f), z=torch.empty(8, dtype=torch.bfloat16, device=device))
 
     @staticmethod
     def alloc(shape: CShape, device="cuda") -> "Saved":
@@ -259,6 +273,61 @@ def sample_draft(h, W_head, E, W_g, n: int, *, uniform: Optional[torch.Tensor] =
                                 ctypes.c_float(temperature), topk, _ptr(res["draft"]), _ptr(res["logp_joint"]),
                                 _ptr(res["topk_tokens"]), _ptr(res["topk_logp"]), _ptr(workspace), workspace.numel(),
                                 _ptr(dev_status), _stream())
+    _check(rc)
+    return res
+
+
+def _shape_full(h, W_full, W_g, x, aux_coef) -> CShape:
+    N, d = h.shape
+    K, V, d2 = W_full.shape
+    n, r = x.shape[1], W_g.shape[0]
+    assert K == n * r and d2 == d and W_g.shape[1] == d and x.shape[0] == N
+    for t in (h, W_full, W_g):
+        assert t.dtype == torch.bfloat16 and t.is_contiguous()
+    assert x.dtype == torch.int32 and x.is_contiguous()
+    return make_shape(N, d, V, n, r, aux_coef)
+
+
+def forward_full(h, W_full, W_g, x, *, aux_coef: Optional[float] = None, saved: Optional[Saved] = None,
+                 want_prefix: bool = False, workspace: Optional[torch.Tensor] = None,
+                 dev_status: Optional[torch.Tensor] = None, out: Optional[dict] = None) -> dict:
+    """cpmtp_forward_full (W_full [n*r, V, d]); returns {"logp", "loss", "counts"[, "logp_prefix"]}."""
+    lib = load_library()
+    shape = _shape_full(h, W_full, W_g, x, aux_coef)
+    dev = h.device
+    if workspace is None:
+        workspace = alloc_workspace(workspace_bytes(shape, OP_FORWARD_FULL), dev)
+    res = out if out is not None else {}
+    res.setdefault("logp", torch.empty(shape.N, dtype=torch.float32, device=dev))
+    res.setdefault("loss", torch.empty(1, dtype=torch.float32, device=dev))
+    res.setdefault("counts", torch.empty(shape.r, dtype=torch.int32, device=dev))
+    if want_prefix:
+        res.setdefault("logp_prefix", torch.empty((shape.N, shape.n), dtype=torch.float32, device=dev))
+    cs = saved.c_struct() if saved is not None else None
+    rc = lib.cpmtp_forward_full(ctypes.byref(shape), _ptr(h), _ptr(W_full), _ptr(W_g), _ptr(x), _ptr(res["logp"]),
+                                _ptr(res["loss"]), _ptr(res.get("logp_prefix")) if want_prefix else None,
+                                ctypes.byref(cs) if cs is not None else None, _ptr(res["counts"]), _ptr(workspace),
+                                workspace.numel(), _ptr(dev_status), _stream())
+    _check(rc)
+    return res
+
+
+def backward_full(h, W_full, W_g, x, saved: Saved, *, aux_coef: Optional[float] = None,
+                  dloss_dlogp: Optional[torch.Tensor] = None, workspace: Optional[torch.Tensor] = None,
+                  dev_status: Optional[torch.Tensor] = None, out: Optional[dict] = None) -> dict:
+    """cpmtp_backward_full; returns {"dh", "dW_full", "dW_g"} (bf16 device tensors)."""
+    lib = load_library()
+    shape = _shape_full(h, W_full, W_g, x, aux_coef)
+    if workspace is None:
+        workspace = alloc_workspace(workspace_bytes(shape, OP_BACKWARD_FULL), h.device)
+    res = out if out is not None else {}
+    for name, ref in (("dh", h), ("dW_full", W_full), ("dW_g", W_g)):
+        if name not in res:
+            res[name] = torch.empty_like(ref)
+    cs = saved.c_struct()
+    rc = lib.cpmtp_backward_full(ctypes.byref(shape), _ptr(h), _ptr(W_full), _ptr(W_g), _ptr(x), ctypes.byref(cs),
+                                 _ptr(dloss_dlogp), _ptr(res["dh"]), _ptr(res["dW_full"]), _ptr(res["dW_g"]),
+                                 _ptr(workspace), workspace.numel(), _ptr(dev_status), _stream())
     _check(rc)
     return res
 

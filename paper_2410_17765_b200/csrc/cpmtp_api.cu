@@ -207,6 +207,71 @@ struct ProfScope {
   }
 };
 
+// ---- full head (Eq. 6 as printed) ----
+struct FullLayout {
+  size_t logw, q, wbar, lse, tgt, part_m, part_l, total;
+  Sched sched;
+  int K, tph, sph;
+  bool wide;
+};
+
+FullLayout full_layout(const cpmtp_shape& s, int sms) {
+  FullLayout L;
+  L.K = s.n * s.r;
+  L.wide = use_wide(s.N, s.d);
+  const int bm = L.wide ? kWideBM : kBM;
+  const int m_tiles = (s.N + bm - 1) / bm;
+  L.tph = (s.V + kBN - 1) / kBN;
+  L.sph = (L.tph + 15) / 16;             // units of at most 16 column tiles
+  int group = static_cast<int>(((L.wide ? 24ll : 64ll) << 20) / (2ll * bm * s.d));
+  if (group < 1) group = 1;
+  L.sched = make_sched(m_tiles, L.K * L.tph, L.K * L.sph, group, s.d / kBK);
+  L.sched.seg_tiles = L.tph;
+  L.sched.seg_stride = s.V;
+  (void)sms;
+  size_t off = 0;
+  auto take = [&](size_t bytes) { size_t o = off; off = align_up(off + bytes); return o; };
+  L.logw = take(sizeof(float) * s.N * s.r);
+  L.q = take(sizeof(float) * s.N * s.r);
+  L.wbar = take(sizeof(float) * CPMTP_MAX_R);
+  L.lse = take(sizeof(float) * static_cast<size_t>(s.N) * L.K);
+  L.tgt = take(sizeof(float) * static_cast<size_t>(s.N) * L.K);
+  L.part_m = take(sizeof(float) * static_cast<size_t>(s.N) * L.K * L.sph);
+  L.part_l = take(sizeof(float) * static_cast<size_t>(s.N) * L.K * L.sph);
+  L.total = off;
+  return L;
+}
+
+struct FullBwdLayout {
+  size_t coef, dg, G, dh32, dwg_part, total;
+  int K, ldv, heads_per_chunk, dwg_slices, dwg_rows_per_slice;
+};
+
+FullBwdLayout full_bwd_layout(const cpmtp_shape& s) {
+  FullBwdLayout L;
+  L.K = s.n * s.r;
+  L.ldv = (s.V + 63) / 64 * 64;
+  long long heads = static_cast<long long>(kLogitGradBudgetBytes / (2ull * s.N * L.ldv));
+  if (const char* env = std::getenv("CPMTP_BWD_CHUNK_HEADS")) {   // testing knob
+    const long long v = std::atoll(env);
+    if (v >= 1) heads = v;
+  }
+  if (heads < 1) heads = 1;
+  if (heads > L.K) heads = L.K;
+  L.heads_per_chunk = static_cast<int>(heads);
+  L.dwg_rows_per_slice = 256;
+  L.dwg_slices = (s.N + L.dwg_rows_per_slice - 1) / L.dwg_rows_per_slice;
+  size_t off = 0;
+  auto take = [&](size_t bytes) { size_t o = off; off = align_up(off + bytes); return o; };
+  L.coef = take(sizeof(float) * s.N * s.r);
+  L.dg = take(sizeof(float) * s.N * s.r);
+  L.G = take(2ull * s.N * L.heads_per_chunk * L.ldv);
+  L.dh32 = take(sizeof(float) * static_cast<size_t>(s.N) * s.d);
+  L.dwg_part = take(sizeof(float) * static_cast<size_t>(L.dwg_slices) * s.r * s.d);
+  L.total = off;
+  return L;
+}
+
 struct SampleLayout {
   FwdLayout fwd;
   size_t logits, z32, lb, part_top, part_best, logp_tmp, total;
@@ -455,6 +520,8 @@ size_t cpmtp_workspace_bytes(const cpmtp_shape* shape, int op) {
     case CPMTP_OP_SCORE: return fwd_layout(*shape, sms).total;
     case CPMTP_OP_BACKWARD: return bwd_layout(*shape).total;
     case CPMTP_OP_SAMPLE: return sample_layout(*shape, sms).total;
+    case CPMTP_OP_FORWARD_FULL: return full_layout(*shape, sms).total;
+    case CPMTP_OP_BACKWARD_FULL: return full_bwd_layout(*shape).total;
     default: return 0;
   }
 }
@@ -538,6 +605,146 @@ int cpmtp_sample_draft(const cpmtp_shape* shape, const void* h, const void* W_he
                                                            part_top, part_best, L.chunks,
                                                            uniform != nullptr ? 1 : 0, step, s.V, s.n, s.r, topk,
                                                            draft, logp_joint, topk_tokens, topk_logp);
+    CPMTP_TRY(cudaGetLastError());
+  }
+  return CPMTP_OK;
+}
+
+int cpmtp_forward_full(const cpmtp_shape* shape, const void* h, const void* W_full, const void* W_g,
+                       const int32_t* x, float* logp, float* loss, float* logp_prefix, const cpmtp_saved* saved,
+                       int32_t* expert_counts, void* workspace, size_t workspace_bytes, int32_t* dev_status,
+                       cpmtp_stream stream) {
+  DeviceInfo* di = nullptr;
+  const int rc = check_common(shape, h, W_full, W_full, W_g, x, workspace, &di);
+  if (rc != CPMTP_OK) return rc;
+  if (logp == nullptr) return CPMTP_ERR_NULL;
+  if (static_cast<double>(shape->n) * shape->r * shape->V >= 2147483648.0) return CPMTP_ERR_SHAPE;
+  if (saved != nullptr && (!saved->lse || !saved->tgt || !saved->logw || !saved->q || !saved->wbar))
+    return CPMTP_ERR_NULL;
+  const cpmtp_shape& s = *shape;
+  const FullLayout L = full_layout(s, di->sms);
+  if (workspace_bytes < L.total) return CPMTP_ERR_WORKSPACE;
+  cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
+  uint8_t* ws = static_cast<uint8_t*>(workspace);
+  float* logw = saved ? saved->logw : reinterpret_cast<float*>(ws + L.logw);
+  float* q = saved ? saved->q : reinterpret_cast<float*>(ws + L.q);
+  float* wbar = saved ? saved->wbar : reinterpret_cast<float*>(ws + L.wbar);
+  float* lse = saved ? saved->lse : reinterpret_cast<float*>(ws + L.lse);
+  float* tgt = saved ? saved->tgt : reinterpret_cast<float*>(ws + L.tgt);
+  float* part_m = reinterpret_cast<float*>(ws + L.part_m);
+  float* part_l = reinterpret_cast<float*>(ws + L.part_l);
+  {
+    ProfScope prof(CPMTP_STAGE_LSE, st);
+    EpiLseFull<kBN>::Params ep{part_m, part_l, tgt, x, dev_status, s.N, s.V, L.K, s.n, s.r, L.tph, L.K * L.sph};
+    const uint64_t b_rows = static_cast<uint64_t>(L.K) * s.V;
+    if (L.wide) {
+      CPMTP_TRY((launch_gemm<WideKK, EpiLseFull<kBN>>(h, s.N, s.d, W_full, b_rows, s.d, s.d, L.sched, ep, dev_status, di->sms, st)));
+    } else {
+      CPMTP_TRY((launch_gemm<CfgKK, EpiLseFull<kBN>>(h, s.N, s.d, W_full, b_rows, s.d, s.d, L.sched, ep, dev_status, di->sms, st)));
+    }
+  }
+  {
+    ProfScope prof(CPMTP_STAGE_MIXTURE, st);
+    const int threads = s.N <= 256 ? 1024 : 256;
+    // the target logits are complete already: handed over as one "partial" per head
+    gate_mixture_kernel<<<s.N, threads, 0, st>>>(static_cast<const uint16_t*>(h), static_cast<const uint16_t*>(W_g),
+                                                s.d, part_m, part_l, L.sph, tgt, 1, logw, lse, nullptr, q, logp,
+                                                logp_prefix, s.N, s.n, s.r);
+    CPMTP_TRY(cudaGetLastError());
+  }
+  if (loss != nullptr || expert_counts != nullptr || saved != nullptr) {
+    ProfScope prof(CPMTP_STAGE_FINALIZE, st);
+    const float aux = (s.flags & CPMTP_FLAG_AUX) ? s.aux_coef : 0.f;
+    finalize_kernel<<<1, 1024, 0, st>>>(logp, logw, wbar, expert_counts, loss, s.N, s.r, aux);
+    CPMTP_TRY(cudaGetLastError());
+  }
+  return CPMTP_OK;
+}
+
+int cpmtp_backward_full(const cpmtp_shape* shape, const void* h, const void* W_full, const void* W_g,
+                        const int32_t* x, const cpmtp_saved* saved, const float* dloss_dlogp, void* dh,
+                        void* dW_full, void* dW_g, void* workspace, size_t workspace_bytes, int32_t* dev_status,
+                        cpmtp_stream stream) {
+  DeviceInfo* di = nullptr;
+  const int rc = check_common(shape, h, W_full, W_full, W_g, x, workspace, &di);
+  if (rc != CPMTP_OK) return rc;
+  if (saved == nullptr || !saved->lse || !saved->logw || !saved->q || !saved->wbar || !dh || !dW_full || !dW_g)
+    return CPMTP_ERR_NULL;
+  if (!aligned(dh, 16) || !aligned(dW_full, 16) || !aligned(dW_g, 16)) return CPMTP_ERR_ALIGN;
+  if (static_cast<double>(shape->n) * shape->r * shape->V >= 2147483648.0) return CPMTP_ERR_SHAPE;
+  const cpmtp_shape& s = *shape;
+  const FullBwdLayout L = full_bwd_layout(s);
+  if (workspace_bytes < L.total) return CPMTP_ERR_WORKSPACE;
+  cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
+  uint8_t* ws = static_cast<uint8_t*>(workspace);
+  float* coef = reinterpret_cast<float*>(ws + L.coef);
+  float* dg = reinterpret_cast<float*>(ws + L.dg);
+  uint16_t* G = reinterpret_cast<uint16_t*>(ws + L.G);
+  float* dh32 = reinterpret_cast<float*>(ws + L.dh32);
+  float* dwg_part = reinterpret_cast<float*>(ws + L.dwg_part);
+  const uint16_t* Wf = static_cast<const uint16_t*>(W_full);
+  const uint16_t* hb = static_cast<const uint16_t*>(h);
+  const int sms = di->sms;
+  const int K = L.K, d = s.d, V = s.V;
+  const float aux = (s.flags & CPMTP_FLAG_AUX) ? s.aux_coef : 0.f;
+  {
+    ProfScope prof(CPMTP_STAGE_COEFF, st);
+    coeff_kernel<<<(s.N + 255) / 256, 256, 0, st>>>(saved->q, saved->logw, saved->wbar, dloss_dlogp, coef, dg, s.N,
+                                                   s.r, aux);
+    CPMTP_TRY(cudaGetLastError());
+  }
+  const bool wide = use_wide(s.N, d);
+  const int bm = wide ? kWideBM : kBM;
+  const int tph = (V + kBN - 1) / kBN;
+  for (int k0 = 0; k0 < K; k0 += L.heads_per_chunk) {
+    const int heads = (K - k0) < L.heads_per_chunk ? (K - k0) : L.heads_per_chunk;
+    const int ldg = L.heads_per_chunk * L.ldv;
+    // recompute the logits of these heads -> G (bf16)
+    {
+      ProfScope prof(CPMTP_STAGE_LOGIT_GRAD, st);
+      EpiLogitGradFull<kBN>::Params ep{G, saved->lse, coef, x, s.N, V, K, s.n, s.r, tph, L.ldv, ldg, k0};
+      Sched sc = make_sched((s.N + bm - 1) / bm, heads * tph, heads * tph, 2048 / bm, d / kBK);
+      sc.seg_tiles = tph;
+      sc.seg_stride = V;
+      const uint16_t* Wc = Wf + static_cast<size_t>(k0) * V * d;
+      const uint64_t b_rows = static_cast<uint64_t>(heads) * V;
+      if (wide) {
+        CPMTP_TRY((launch_gemm<WideKK, EpiLogitGradFull<kBN>>(hb, s.N, d, Wc, b_rows, d, d, sc, ep, dev_status, sms, st)));
+      } else {
+        CPMTP_TRY((launch_gemm<CfgKK, EpiLogitGradFull<kBN>>(hb, s.N, d, Wc, b_rows, d, d, sc, ep, dev_status, sms, st)));
+      }
+    }
+    for (int k = k0; k < k0 + heads; ++k) {
+      const uint16_t* Gk = G + static_cast<size_t>(k - k0) * L.ldv;
+      const uint16_t* Wk = Wf + static_cast<size_t>(k) * V * d;
+      // dW_full[k][V, d] = G_k^T[V, N] * h[N, d]
+      {
+        ProfScope prof(CPMTP_STAGE_DE, st);
+        EpiStoreBf16<kBN, false>::Params ep{static_cast<uint16_t*>(dW_full) + static_cast<size_t>(k) * V * d, nullptr,
+                                            nullptr, V, d, d, 0};
+        CPMTP_TRY((gemm_auto<true, true, EpiStoreBf16<kBN, false>>(Gk, ldg, hb, d, V, d, s.N, 2048, ep, dev_status, sms, st)));
+      }
+      // dh (+)= G_k[N, V] * W_full[k][V, d]
+      {
+        ProfScope prof(CPMTP_STAGE_DH, st);
+        EpiAccumF32<kBN>::Params ep{dh32, s.N, d, d, k > 0 ? 1 : 0};
+        CPMTP_TRY((gemm_auto<false, true, EpiAccumF32<kBN>>(Gk, ldg, Wk, d, s.N, d, V, 2048, ep, dev_status, sms, st)));
+      }
+    }
+  }
+  {
+    ProfScope prof(CPMTP_STAGE_DE_CONVERT, st);
+    const size_t total = static_cast<size_t>(s.N) * d;
+    dh_finish_kernel<<<static_cast<unsigned>((total + 255) / 256), 256, 0, st>>>(
+        dh32, dg, static_cast<const uint16_t*>(W_g), static_cast<uint16_t*>(dh), s.N, d, s.r);
+    CPMTP_TRY(cudaGetLastError());
+  }
+  {
+    ProfScope prof(CPMTP_STAGE_DW_G, st);
+    dim3 grid((d + 127) / 128, L.dwg_slices);
+    dwg_partial_kernel<CPMTP_MAX_R><<<grid, 128, 0, st>>>(dg, hb, dwg_part, s.N, d, s.r, L.dwg_rows_per_slice);
+    CPMTP_TRY(cudaGetLastError());
+    dwg_reduce_kernel<<<(s.r * d + 255) / 256, 256, 0, st>>>(dwg_part, static_cast<uint16_t*>(dW_g), L.dwg_slices, s.r, d);
     CPMTP_TRY(cudaGetLastError());
   }
   return CPMTP_OK;

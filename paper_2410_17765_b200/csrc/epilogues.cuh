@@ -179,6 +179,86 @@ struct EpiLse {
 };
 
 // ---------------------------------------------------------------------------
+// Full head (Eq. 6 as printed: one unembedding per (token, expert)): the logits of all heads come
+// from ONE GEMM  S[i, k*V + v] = W_full[k][v, :] . h[i, :]  whose column tiles are segmented by head.
+// A unit stays inside one head; each thread keeps the running (max, sum-exp) of its row for that
+// head, and picks the target logit straight from the fp32 accumulator when its column comes by.
+template <int BN>
+struct EpiLseFull {
+  struct Params {
+    float* part_m;       // [M, K * sph]  (sph = splits per head)
+    float* part_l;
+    float* tgt;          // [M, K]
+    const int32_t* x;    // [M, n]
+    int* dev_status;
+    int M, V, K, n, r, tph, n_splits;   // tph = column tiles per head
+  };
+  struct State { float m2, l, tgt; int k, tok; };
+  static constexpr int SMEM_BYTES = 0;
+  __device__ static void unit_begin(const Params&, State& st, int, int, int) {
+    st.m2 = -INFINITY;
+    st.l = 0.f;
+    st.tgt = 0.f;
+    st.k = -1;
+    st.tok = -1;
+  }
+  __device__ static void unit_end(const Params& p, State& st, int m_tile, int split, int row_in_tile, uint8_t*, int) {
+    const int row = m_tile * kBM + row_in_tile;
+    if (row < p.M && st.k >= 0) {
+      p.part_m[static_cast<size_t>(row) * p.n_splits + split] = st.m2;
+      p.part_l[static_cast<size_t>(row) * p.n_splits + split] = st.l;
+      if (st.tok == -2) p.tgt[static_cast<size_t>(row) * p.K + st.k] = st.tgt;   // this unit held the target column
+    }
+  }
+  __device__ static void tile(const Params& p, State& st, uint32_t tacc, int m_tile, int n_tile, int row_in_tile,
+                              uint8_t*, int) {
+    const int row = m_tile * kBM + row_in_tile;
+    const int k = n_tile / p.tph;
+    const int local0 = (n_tile - k * p.tph) * BN;
+    if (st.k != k) {   // first tile of the unit (units never straddle heads)
+      st.k = k;
+      if (row < p.M) {
+        int tok = p.x[static_cast<size_t>(row) * p.n + k / p.r];
+        if (tok < 0 || tok >= p.V) {
+          if (p.dev_status != nullptr) atomicMax(p.dev_status, kDevTargetOutOfRange);
+          tok = tok < 0 ? 0 : p.V - 1;
+        }
+        st.tok = tok;
+      }
+    }
+#pragma unroll 1
+    for (int c = 0; c < BN; c += 32) {
+      const int col0 = local0 + c;
+      if (col0 >= p.V) break;   // uniform across the CTA
+      float v[32];
+      ptx::tmem_ld_32x32(tacc + c, v);
+      ptx::tmem_ld_wait();
+      const int t = st.tok - col0;
+      if (t >= 0 && t < 32) {
+#pragma unroll
+        for (int j = 0; j < 32; ++j)
+          if (j == t) st.tgt = v[j];
+        st.tok = -2;
+      }
+      if (col0 + 32 > p.V) {
+#pragma unroll
+        for (int j = 0; j < 32; ++j)
+          if (col0 + j >= p.V) v[j] = -INFINITY;
+      }
+      float cm = v[0];
+#pragma unroll
+      for (int j = 1; j < 32; ++j) cm = fmaxf(cm, v[j]);
+      const float m_new = fmaxf(st.m2, cm * kLog2e);
+      float sum = 0.f;
+#pragma unroll
+      for (int j = 0; j < 32; ++j) sum += ptx::ex2_approx(fmaf(v[j], kLog2e, -m_new));
+      st.l = st.l * ptx::ex2_approx(st.m2 - m_new) + sum;
+      st.m2 = m_new;
+    }
+  }
+};
+
+// ---------------------------------------------------------------------------
 // Backward: recompute a logits tile and turn it into the logit gradient
 //   G[(i,k), v] = c[i, alpha(k)] * (1[v = x[i, s(k)]] - exp(S - lse[i,k]))
 // (derivative of Eq. 9 through Eq. 8), stored as bf16 for the two GEMMs that
@@ -238,6 +318,68 @@ struct EpiLogitGrad {
           if (col0 + j >= p.V) v[j] = 0.f;
       }
       if (valid) store_bf16x32(p.G + static_cast<size_t>(row) * p.ldg + col0, v);
+    }
+  }
+};
+
+// ---------------------------------------------------------------------------
+// Full head, backward: the logit gradient of a few heads [k0, k0 + heads) at a time,
+//   G[i, (k - k0) * ldv + v] = c[i, alpha(k)] * (1[v = x[i, s(k)]] - exp(S[i,k,v] - lse[i,k])),
+// from the same segmented GEMM as the forward.  Columns in [V, ldv) of every head are zero.
+template <int BN>
+struct EpiLogitGradFull {
+  struct Params {
+    uint16_t* G;          // [M, ldg] bf16, ldg = heads * ldv
+    const float* lse;     // [M, K]
+    const float* coef;    // [M, r]
+    const int32_t* x;     // [M, n]
+    int M, V, K, n, r, tph, ldv, ldg, k0;
+  };
+  struct State { float lse2, coef; int tok, k; };
+  static constexpr int SMEM_BYTES = 0;
+  __device__ static void unit_begin(const Params&, State& st, int, int, int) { st.k = -1; }
+  __device__ static void unit_end(const Params&, State&, int, int, int, uint8_t*, int) {}
+  __device__ static void tile(const Params& p, State& st, uint32_t tacc, int m_tile, int n_tile, int row_in_tile,
+                              uint8_t*, int) {
+    const int row = m_tile * kBM + row_in_tile;
+    const bool valid = row < p.M;
+    const int k_local = n_tile / p.tph;
+    const int local0 = (n_tile - k_local * p.tph) * BN;
+    const int k = p.k0 + k_local;
+    if (st.k != k) {
+      st.k = k;
+      st.lse2 = 0.f;
+      st.coef = 0.f;
+      st.tok = -1;
+      if (valid) {
+        st.lse2 = p.lse[static_cast<size_t>(row) * p.K + k] * kLog2e;
+        st.coef = p.coef[static_cast<size_t>(row) * p.r + (k % p.r)];
+        const int tok = p.x[static_cast<size_t>(row) * p.n + k / p.r];
+        st.tok = tok < 0 ? 0 : (tok >= p.V ? p.V - 1 : tok);
+      }
+    }
+    const float nc = -st.coef;
+#pragma unroll 1
+    for (int c = 0; c < BN; c += 32) {
+      const int col0 = local0 + c;
+      if (col0 >= p.ldv) break;
+      float v[32];
+      ptx::tmem_ld_32x32(tacc + c, v);
+      ptx::tmem_ld_wait();
+#pragma unroll
+      for (int j = 0; j < 32; ++j) v[j] = nc * ptx::ex2_approx(fmaf(v[j], kLog2e, -st.lse2));
+      const int t = st.tok - col0;
+      if (t >= 0 && t < 32) {
+#pragma unroll
+        for (int j = 0; j < 32; ++j)
+          if (j == t) v[j] += st.coef;
+      }
+      if (col0 + 32 > p.V) {
+#pragma unroll
+        for (int j = 0; j < 32; ++j)
+          if (col0 + j >= p.V) v[j] = 0.f;
+      }
+      if (valid) store_bf16x32(p.G + static_cast<size_t>(row) * p.ldg + static_cast<size_t>(k_local) * p.ldv + col0, v);
     }
   }
 };

@@ -218,6 +218,18 @@ __global__ void dwg_reduce_kernel(const float* __restrict__ part, uint16_t* __re
   dW_g[idx] = static_cast<uint16_t>(ptx::pack_bf16x2(acc, 0.f) & 0xFFFFu);
 }
 
+// dh[i, :] = bf16( acc[i, :] + sum_b dg[i, b] * W_g[b, :] ): the gate path of Eq. 7 added to an fp32 sum.
+__global__ void dh_finish_kernel(const float* __restrict__ acc, const float* __restrict__ dg,
+                                 const uint16_t* __restrict__ W_g, uint16_t* __restrict__ dh, int N, int d, int r) {
+  const size_t idx = static_cast<size_t>(blockIdx.x) * blockDim.x + threadIdx.x;
+  if (idx >= static_cast<size_t>(N) * d) return;
+  const int i = static_cast<int>(idx / d), j = static_cast<int>(idx - static_cast<size_t>(i) * d);
+  float v = acc[idx];
+  for (int b = 0; b < r; ++b)
+    v = fmaf(dg[static_cast<size_t>(i) * r + b], __uint_as_float(static_cast<uint32_t>(W_g[static_cast<size_t>(b) * d + j]) << 16), v);
+  dh[idx] = static_cast<uint16_t>(ptx::pack_bf16x2(v, 0.f) & 0xFFFFu);
+}
+
 __global__ void f32_to_bf16_kernel(const float* __restrict__ src, uint16_t* __restrict__ dst, size_t count) {
   const size_t stride = static_cast<size_t>(gridDim.x) * blockDim.x * 4;
   for (size_t i = (static_cast<size_t>(blockIdx.x) * blockDim.x + threadIdx.x) * 4; i < count; i += stride) {

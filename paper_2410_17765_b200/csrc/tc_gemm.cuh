@@ -48,6 +48,12 @@ struct Sched {
   int m_group;    // row tiles that are swept together (L2 locality)
   int k_blocks;   // contraction length / 64, rounded up
   int units;      // ceil(m_tiles / m_group) * m_group * n_splits
+  // Segmented columns (0 = off): the B rows form segments of seg_stride rows, each covered by
+  // seg_tiles column tiles that start at the segment's first row (the last tile of a segment
+  // may run into the next one; the epilogue masks it).  Column tile nt then starts at B row
+  // (nt / seg_tiles) * seg_stride + (nt % seg_tiles) * BN instead of nt * BN.
+  int seg_tiles;
+  int seg_stride;
 };
 
 inline Sched make_sched(int m_tiles, int n_tiles, int n_splits, int m_group, int k_blocks) {
@@ -62,6 +68,8 @@ inline Sched make_sched(int m_tiles, int n_tiles, int n_splits, int m_group, int
   s.m_group = m_group;
   s.k_blocks = k_blocks;
   s.units = ((m_tiles + m_group - 1) / m_group) * m_group * n_splits;
+  s.seg_tiles = 0;
+  s.seg_stride = 0;
   return s;
 }
 
@@ -176,6 +184,9 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         int m_tile, split, n_begin, n_end;
         if (!decode_unit(sched, u, m_tile, split, n_begin, n_end)) continue;
         for (int nt = n_begin; nt < n_end && alive; ++nt) {
+          const int b_row0 = sched.seg_tiles > 0
+                                 ? (nt / sched.seg_tiles) * sched.seg_stride + (nt % sched.seg_tiles) * Cfg::BN
+                                 : nt * Cfg::BN;
           for (int kb = 0; kb < sched.k_blocks; ++kb, ++it) {
             const int s = it % Cfg::STAGES;
             const uint32_t ph = (it / Cfg::STAGES) & 1;
@@ -192,11 +203,11 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                 ptx::tma_load_2d(a_dst + j * 8192, &tmA, full_bar(s), m_tile * Cfg::TILE_M + j * 64, kb * kBK);
             }
             if constexpr (!Cfg::B_MN) {
-              ptx::tma_load_2d(b_dst, &tmB, full_bar(s), kb * kBK, nt * Cfg::BN);
+              ptx::tma_load_2d(b_dst, &tmB, full_bar(s), kb * kBK, b_row0);
             } else {
 #pragma unroll
               for (int j = 0; j < Cfg::BN / 64; ++j)
-                ptx::tma_load_2d(b_dst + j * 8192, &tmB, full_bar(s), nt * Cfg::BN + j * 64, kb * kBK);
+                ptx::tma_load_2d(b_dst + j * 8192, &tmB, full_bar(s), b_row0 + j * 64, kb * kBK);
             }
           }
         }

@@ -45,6 +45,8 @@ CONFIGS = {
     # train_fwd_bwd at 1/16 of the positions: same kernels and tile shapes, small enough to profile
     "train_fwd_bwd_small": Shape(N=512, d=4096, V=32000, n=4, r=8),
     # bigvocab at 1/4 of the positions (forward only): same schedule regime, profilable
+    # full-head variant (Eq. 6 as printed): W_full is n*r*V*d = 1 GB here
+    "full_head_train": Shape(N=4096, d=2048, V=32000, n=2, r=4),
     "bigvocab_fwd_small": Shape(N=2048, d=4096, V=128256, n=4, r=16),
 }
 
@@ -122,6 +124,13 @@ def make_inputs(
     else:
         raise ValueError(f"unknown target distribution {targets!r}")
     return Inputs(shape=s, h=h, W_head=W_head, E=E, W_g=W_g, x=x)
+
+
+def make_full_head(shape: Shape, seed: int = 0, *, weight_std: float = 0.02, weight_scale: float = 1.0) -> torch.Tensor:
+    """W_full [n*r, V, d] bf16 for the full-head variant: one N(0, std) unembedding per (token, expert)."""
+    gen = torch.Generator(device="cpu")
+    gen.manual_seed(seed + 7919)
+    return _randn_bf16(gen, (shape.K, shape.V, shape.d), weight_std * weight_scale)
 
 
 def subsample_positions(inp: Inputs, idx: torch.Tensor) -> Inputs:

@@ -1,0 +1,85 @@
+"""GPU parity of the full-head variant (cpmtp_forward_full / cpmtp_backward_full) against the oracle."""
+import os
+
+import numpy as np
+import pytest
+import torch
+
+from oracle import cp_head
+from paper_2410_17765_b200 import synth
+
+pytestmark = pytest.mark.gpu
+
+LOGP_TOL = 2e-3
+GRAD_TOL = 1e-2
+
+
+def rel_l2(a, b):
+    a = np.asarray(a, dtype=np.float64)
+    b = np.asarray(b, dtype=np.float64)
+    return float(np.linalg.norm(a - b) / max(np.linalg.norm(b), 1e-300))
+
+
+SHAPES = {
+    "ragged": synth.Shape(N=70, d=320, V=1000, n=2, r=3),      # V % 256 != 0: head tiles run into the next head
+    "tiny": synth.Shape(N=64, d=256, V=1024, n=3, r=4),
+    "small_v": synth.Shape(N=200, d=128, V=77, n=4, r=2),
+    "rank1": synth.Shape(N=33, d=64, V=300, n=3, r=1),
+    "many_rows": synth.Shape(N=1100, d=4096, V=520, n=1, r=2),   # wide tiles (rows >= 512, d >= 4096)
+}
+
+
+@pytest.mark.parametrize("name,chunk_heads", [("ragged", None), ("ragged", 2), ("tiny", 5), ("small_v", 1),
+                                              ("rank1", None), ("many_rows", None)])
+def test_full_head_forward_and_backward_match_oracle(name, chunk_heads):
+    from paper_2410_17765_b200 import binding
+
+    shape = SHAPES[name]
+    inp = synth.make_inputs(shape, seed=0)
+    # logits of the shared head have std 0.02^2 * d; give the full head a comparable, non-trivial scale
+    W_full = synth.make_full_head(shape, seed=0, weight_scale=4.0)
+    ref = cp_head.forward_full(inp.h, W_full, inp.W_g, inp.x, shape.n, shape.r, aux_coef=1.0)
+    refg = cp_head.backward_full(inp.h, W_full, inp.W_g, inp.x, shape.n, shape.r, aux_coef=1.0)
+    h, Wf, Wg, x = inp.h.cuda(), W_full.cuda(), inp.W_g.cuda(), inp.x.cuda()
+    cs = binding.make_shape(shape.N, shape.d, shape.V, shape.n, shape.r)
+    saved = binding.Saved.alloc_full(cs)
+    st = torch.zeros(1, dtype=torch.int32, device="cuda")
+    old = os.environ.get("CPMTP_BWD_CHUNK_HEADS")
+    try:
+        if chunk_heads is not None:
+            os.environ["CPMTP_BWD_CHUNK_HEADS"] = str(chunk_heads)
+        out = binding.forward_full(h, Wf, Wg, x, aux_coef=1.0, saved=saved, want_prefix=True, dev_status=st)
+        g = binding.backward_full(h, Wf, Wg, x, saved, aux_coef=1.0, dev_status=st)
+        torch.cuda.synchronize()
+    finally:
+        if old is None:
+            os.environ.pop("CPMTP_BWD_CHUNK_HEADS", None)
+        else:
+            os.environ["CPMTP_BWD_CHUNK_HEADS"] = old
+    assert int(st.item()) == 0
+    assert np.max(np.abs(out["logp"].cpu().numpy() - ref.logp)) <= LOGP_TOL
+    assert abs(float(out["loss"].item()) - ref.loss) <= LOGP_TOL
+    assert np.max(np.abs(out["logp_prefix"].cpu().numpy() - cp_head.prefix_log_probs(ref))) <= LOGP_TOL
+    assert np.max(np.abs(saved.lse.cpu().numpy() - ref.lse)) <= 1e-3
+    assert np.max(np.abs(saved.tgt.cpu().numpy() - ref.tgt)) <= 1e-3 * max(1.0, np.abs(ref.tgt).max())
+    assert int(out["counts"].sum().item()) == shape.N
+    for key, want in (("dh", refg.dh), ("dW_full", refg.dW_full), ("dW_g", refg.dW_g)):
+        got = g[key].float().cpu().numpy()
+        if np.linalg.norm(want) == 0:
+            assert np.abs(got).max() == 0, key
+        else:
+            assert rel_l2(got, want) <= GRAD_TOL, (key, rel_l2(got, want))
+
+
+def test_full_head_reduces_to_the_shared_head_library_path():
+    """W_full[k] = bf16(E . W_head[k]) run through the full-head path agrees with the shared-head path."""
+    from paper_2410_17765_b200 import binding
+
+    shape = synth.Shape(N=96, d=256, V=900, n=2, r=4)
+    inp = synth.make_inputs(shape, seed=3, weight_scale=3.0)
+    W_full = torch.stack([(inp.E.double() @ inp.W_head[k].double()).to(torch.bfloat16) for k in range(shape.K)])
+    a = binding.forward(inp.h.cuda(), inp.W_head.cuda(), inp.E.cuda(), inp.W_g.cuda(), inp.x.cuda())
+    b = binding.forward_full(inp.h.cuda(), W_full.contiguous().cuda(), inp.W_g.cuda(), inp.x.cuda())
+    torch.cuda.synchronize()
+    # the only difference is where bf16 rounding happens (z vs the product matrix)
+    assert float((a["logp"] - b["logp"]).abs().max()) <= 2e-2
