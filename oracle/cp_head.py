@@ -328,3 +328,37 @@ def backward_full(h, W_full, W_g, x, n: int, r: int, *, aux_coef: float = 0.0, d
         dW_full[k] = G.T @ hd
         dh += G @ Wk
     return GradientsFull(dh=dh, dW_full=dW_full, dW_g=dW_g)
+
+
+def accepted_prefix_greedy(draft_tokens, base_tokens) -> np.ndarray:
+    """Draft-then-verify with greedy decoding (Preliminaries): the number of leading draft tokens that
+    equal the base model's tokens, i.e. the length of the longest common prefix, per position."""
+    d, b = _i64(draft_tokens), _i64(base_tokens)
+    out = np.zeros(d.shape[0], dtype=np.int64)
+    for i in range(d.shape[0]):
+        k = 0
+        while k < d.shape[1] and d[i, k] == b[i, k]:
+            k += 1
+        out[i] = k
+    return out
+
+
+def accepted_prefix_sampled(logp_draft_prefix, logp_base, uniform) -> np.ndarray:
+    """Probabilistic verification (the generalisation the Preliminaries mention): draft token s, drawn
+    with conditional probability q_s = exp(prefix[s] - prefix[s-1]), is kept with probability
+    min(1, p_s / q_s), p_s = exp(logp_base[s]) the base model's probability of that token; the accepted
+    length is the number of tokens kept before the first rejection (uniform[i, s] decides token s)."""
+    pre, lb, u = _f64(logp_draft_prefix), _f64(logp_base), _f64(uniform)
+    N, n = pre.shape
+    out = np.zeros(N, dtype=np.int64)
+    for i in range(N):
+        k = 0
+        prev = 0.0
+        while k < n:
+            logq = pre[i, k] - prev
+            if not (u[i, k] < min(1.0, np.exp(lb[i, k] - logq))):
+                break
+            prev = pre[i, k]
+            k += 1
+        out[i] = k
+    return out
