@@ -191,6 +191,22 @@ int cpmtp_backward_full(const cpmtp_shape* shape, const void* h, const void* W_f
                         size_t workspace_bytes, int32_t* dev_status, cpmtp_stream stream);
 
 /*
+ * Verify drafts (draft-then-verify of the Preliminaries; speculative-decoding section).
+ * accepted [N] int32 out: how many leading tokens of each draft are kept.
+ *  - Greedy (base_tokens != NULL): the longest common prefix of draft [N,n] and the
+ *    base model's tokens base_tokens [N,n].
+ *  - Probabilistic (base_tokens == NULL): token s of a draft is kept with probability
+ *    min(1, p_s / q_s), where q_s = exp(logp_prefix[i,s] - logp_prefix[i,s-1]) is the
+ *    probability the CP head gave it (logp_prefix [N,n] as returned by
+ *    cpmtp_score_draft) and p_s = exp(logp_base[i,s]) the base model's; uniform [N,n]
+ *    in [0,1) decides; counting stops at the first rejection.
+ * All pointers are device pointers; no workspace is needed.
+ */
+int cpmtp_verify_draft(int32_t N, int32_t n, const int32_t* draft, const int32_t* base_tokens,
+                       const float* logp_prefix, const float* logp_base, const float* uniform,
+                       int32_t* accepted, cpmtp_stream stream);
+
+/*
  * cpmtp_score_draft for callers that cannot hand over scratch memory.  Code that
  * runs where device allocation is off-limits -- inside a serving loop that has
  * frozen its memory pool, in a plugin that is given tensors but no allocator, or

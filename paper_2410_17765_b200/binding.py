@@ -22,7 +22,7 @@ EXPORTS = [
     "cpmtp_version", "cpmtp_status_string", "cpmtp_workspace_bytes", "cpmtp_forward", "cpmtp_backward",
     "cpmtp_score_draft", "cpmtp_host_staging_bytes", "cpmtp_forward_host", "cpmtp_profile_begin",
     "cpmtp_profile_end", "cpmtp_score_draft_static", "cpmtp_sample_draft",
-    "cpmtp_forward_full", "cpmtp_backward_full",
+    "cpmtp_forward_full", "cpmtp_backward_full", "cpmtp_verify_draft",
 ]
 
 STATIC_SCRATCH_BYTES = 4 << 20
@@ -77,6 +77,8 @@ def load_library() -> ctypes.CDLL:
     lib.cpmtp_forward_full.argtypes = [shp, vp, vp, vp, i32p, fp, fp, fp, svp, i32p, vp, sz, i32p, vp]
     lib.cpmtp_backward_full.restype = ctypes.c_int
     lib.cpmtp_backward_full.argtypes = [shp, vp, vp, vp, i32p, svp, fp, vp, vp, vp, vp, sz, i32p, vp]
+    lib.cpmtp_verify_draft.restype = ctypes.c_int
+    lib.cpmtp_verify_draft.argtypes = [ctypes.c_int32, ctypes.c_int32, i32p, i32p, fp, fp, fp, i32p, vp]
     lib.cpmtp_score_draft_static.restype = ctypes.c_int
     lib.cpmtp_score_draft_static.argtypes = [shp, vp, vp, vp, vp, i32p, fp, fp, i32p, vp]
     lib.cpmtp_profile_begin.restype = ctypes.c_int
@@ -330,6 +332,20 @@ def backward_full(h, W_full, W_g, x, saved: Saved, *, aux_coef: Optional[float] 
                                  _ptr(workspace), workspace.numel(), _ptr(dev_status), _stream())
     _check(rc)
     return res
+
+
+def verify_draft(draft: Optional[torch.Tensor] = None, base_tokens: Optional[torch.Tensor] = None, *,
+                 logp_prefix: Optional[torch.Tensor] = None, logp_base: Optional[torch.Tensor] = None,
+                 uniform: Optional[torch.Tensor] = None) -> torch.Tensor:
+    """cpmtp_verify_draft: accepted draft length per position (int32 device tensor).
+    Greedy: pass draft and base_tokens [N, n]; probabilistic: pass logp_prefix, logp_base, uniform [N, n]."""
+    ref = base_tokens if base_tokens is not None else logp_prefix
+    N, n = ref.shape
+    accepted = torch.empty(N, dtype=torch.int32, device=ref.device)
+    rc = load_library().cpmtp_verify_draft(N, n, _ptr(draft), _ptr(base_tokens), _ptr(logp_prefix), _ptr(logp_base),
+                                           _ptr(uniform), _ptr(accepted), _stream())
+    _check(rc)
+    return accepted
 
 
 def score_draft_static(h, W_head, E, W_g, draft, *, want_prefix: bool = True,

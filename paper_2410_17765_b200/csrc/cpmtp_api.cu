@@ -750,6 +750,22 @@ int cpmtp_backward_full(const cpmtp_shape* shape, const void* h, const void* W_f
   return CPMTP_OK;
 }
 
+int cpmtp_verify_draft(int32_t N, int32_t n, const int32_t* draft, const int32_t* base_tokens,
+                       const float* logp_prefix, const float* logp_base, const float* uniform, int32_t* accepted,
+                       cpmtp_stream stream) {
+  if (N < 1 || n < 1 || n > CPMTP_MAX_N) return CPMTP_ERR_SHAPE;
+  if (accepted == nullptr) return CPMTP_ERR_NULL;
+  if (base_tokens != nullptr) {
+    if (draft == nullptr) return CPMTP_ERR_NULL;
+  } else if (!logp_prefix || !logp_base || !uniform) {
+    return CPMTP_ERR_NULL;
+  }
+  verify_draft_kernel<<<(N + 127) / 128, 128, 0, reinterpret_cast<cudaStream_t>(stream)>>>(
+      draft, base_tokens, logp_prefix, logp_base, uniform, accepted, N, n);
+  CPMTP_TRY(cudaGetLastError());
+  return CPMTP_OK;
+}
+
 int cpmtp_score_draft_static(const cpmtp_shape* shape, const void* h, const void* W_head, const void* E,
                              const void* W_g, const int32_t* draft, float* logp_joint, float* logp_prefix,
                              int32_t* dev_status, cpmtp_stream stream) {

@@ -237,4 +237,26 @@ __global__ void draft_step_final_kernel(const float* __restrict__ z32, const uin
   }
 }
 
+// Draft verification: one thread per position.
+__global__ void verify_draft_kernel(const int32_t* __restrict__ draft, const int32_t* __restrict__ base_tokens,
+                                    const float* __restrict__ logp_prefix, const float* __restrict__ logp_base,
+                                    const float* __restrict__ uniform, int32_t* __restrict__ accepted, int N, int n) {
+  const int i = blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= N) return;
+  int k = 0;
+  if (base_tokens != nullptr) {
+    while (k < n && draft[static_cast<size_t>(i) * n + k] == base_tokens[static_cast<size_t>(i) * n + k]) ++k;
+  } else {
+    float prev = 0.f;
+    while (k < n) {
+      const float pre = logp_prefix[static_cast<size_t>(i) * n + k];
+      const float ratio = expf(logp_base[static_cast<size_t>(i) * n + k] - (pre - prev));
+      if (!(uniform[static_cast<size_t>(i) * n + k] < fminf(1.f, ratio))) break;
+      prev = pre;
+      ++k;
+    }
+  }
+  accepted[i] = k;
+}
+
 }  // namespace cpmtp

@@ -107,3 +107,27 @@ def test_draft_is_deterministic_and_validates_arguments():
         binding.sample_draft(*dev, shape.n, topk=9)
     with pytest.raises(binding.CpmtpError):
         binding.sample_draft(*dev, shape.n, uniform=torch.rand((4, 2, 900), device="cuda"), temperature=0.0)
+
+
+def test_verify_draft_matches_oracle():
+    from paper_2410_17765_b200 import binding
+
+    g = torch.Generator().manual_seed(0)
+    N, n = 1000, 4
+    draft = torch.randint(0, 3, (N, n), generator=g, dtype=torch.int32)
+    base = torch.randint(0, 3, (N, n), generator=g, dtype=torch.int32)
+    got = binding.verify_draft(draft.cuda(), base.cuda())
+    assert np.array_equal(got.cpu().numpy(), cp_head.accepted_prefix_greedy(draft, base))
+    # probabilistic rule: draft-side conditionals from cumulative sums, base side arbitrary
+    cond = -torch.rand((N, n), generator=g) * 3
+    pre = torch.cumsum(cond, dim=1).float()
+    lb = (cond + torch.randn((N, n), generator=g)).float()
+    u = torch.rand((N, n), generator=g).float()
+    got = binding.verify_draft(logp_prefix=pre.cuda(), logp_base=lb.cuda(), uniform=u.cuda()).cpu().numpy()
+    want = cp_head.accepted_prefix_sampled(pre, lb, u)
+    # a decision within fp32 rounding of its threshold may go either way: compare where the margin is clear
+    ratio = np.minimum(1.0, np.exp(lb.double().numpy() - np.diff(pre.double().numpy(), axis=1, prepend=0.0)))
+    clear = np.all(np.abs(u.double().numpy() - ratio) > 1e-5, axis=1)
+    assert clear.mean() > 0.99
+    assert np.array_equal(got[clear], want[clear])
+    assert got.min() >= 0 and got.max() <= n
