@@ -405,7 +405,7 @@ int run_forward(const cpmtp_shape& s, const uint16_t* h, const uint16_t* W_head,
   if (loss != nullptr || counts != nullptr || saved != nullptr) {
     ProfScope prof(CPMTP_STAGE_FINALIZE, stream);
     const float aux = (s.flags & CPMTP_FLAG_AUX) ? s.aux_coef : 0.f;
-    finalize_kernel<<<1, 1024, 0, stream>>>(logp, logw, wbar, counts, loss, s.N, s.r, aux);
+    finalize_kernel<<<1, kFinalizeThreads, 0, stream>>>(logp, logw, wbar, counts, loss, s.N, s.r, aux);
     CPMTP_TRY(cudaGetLastError());
   }
   return CPMTP_OK;
@@ -655,7 +655,7 @@ int cpmtp_forward_full(const cpmtp_shape* shape, const void* h, const void* W_fu
   if (loss != nullptr || expert_counts != nullptr || saved != nullptr) {
     ProfScope prof(CPMTP_STAGE_FINALIZE, st);
     const float aux = (s.flags & CPMTP_FLAG_AUX) ? s.aux_coef : 0.f;
-    finalize_kernel<<<1, 1024, 0, st>>>(logp, logw, wbar, expert_counts, loss, s.N, s.r, aux);
+    finalize_kernel<<<1, kFinalizeThreads, 0, st>>>(logp, logw, wbar, expert_counts, loss, s.N, s.r, aux);
     CPMTP_TRY(cudaGetLastError());
   }
   return CPMTP_OK;

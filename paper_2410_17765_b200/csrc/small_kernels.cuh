@@ -113,53 +113,80 @@ __global__ void gate_mixture_kernel(const uint16_t* __restrict__ h, const uint16
   }
 }
 
-// Loss, mean gate weights and hard expert counts (Eq. 10's n_a).  One block.
-//   wbar[a] = (1/N) sum_i exp(logw[i,a]);  counts[a] = #{i : argmax_b w[i,b] = a}
+// Loss, mean gate weights and hard expert counts (Eq. 10's n_a).  One block, one pass:
+//   wbar[a] = (1/N) sum_i exp(logw[i,a]);  counts[a] = #{i : argmax_b w[i,b] = a} (ties -> lowest a)
 //   loss = -(1/N) sum_i logp[i] + aux_coef * sum_a wbar[a]^2
-__global__ void finalize_kernel(const float* __restrict__ logp, const float* __restrict__ logw,
+// Every thread accumulates its positions in double precision; the per-thread sums are then
+// combined in a fixed order (warp shuffles, then across warps), so the result is reproducible.
+constexpr int kFinalizeThreads = 512;
+__global__ void __launch_bounds__(kFinalizeThreads) finalize_kernel(const float* __restrict__ logp, const float* __restrict__ logw,
                                 float* __restrict__ wbar, int* __restrict__ counts,
                                 float* __restrict__ loss, int N, int r, float aux_coef) {
-  __shared__ double red[1024];
-  __shared__ int redi[1024];
-  __shared__ double wbar_s[32];
-  const int t = threadIdx.x;
-  for (int a = 0; a <= r; ++a) {   // a == r: the logp sum
-    double acc = 0.0;
-    int cnt = 0;
-    for (int i = t; i < N; i += blockDim.x) {
+  __shared__ double sum_s[32][CPMTP_MAX_R + 1];
+  __shared__ int cnt_s[32][CPMTP_MAX_R];
+  const int t = threadIdx.x, warp = t >> 5, lane = t & 31, nwarps = blockDim.x >> 5;
+  double acc[CPMTP_MAX_R + 1];
+  int cnt[CPMTP_MAX_R];
+#pragma unroll
+  for (int a = 0; a <= CPMTP_MAX_R; ++a) acc[a] = 0.0;
+#pragma unroll
+  for (int a = 0; a < CPMTP_MAX_R; ++a) cnt[a] = 0;
+  for (int i = t; i < N; i += blockDim.x) {
+    const float* row = logw + static_cast<size_t>(i) * r;
+    float best = -INFINITY;
+    int arg = 0;
+#pragma unroll
+    for (int a = 0; a < CPMTP_MAX_R; ++a) {
       if (a < r) {
-        const float* row = logw + static_cast<size_t>(i) * r;
-        acc += static_cast<double>(expf(row[a]));
-        bool is_max = true;
-        for (int b = 0; b < r; ++b)
-          if (row[b] > row[a] || (row[b] == row[a] && b < a)) is_max = false;
-        cnt += is_max ? 1 : 0;
-      } else {
-        acc += static_cast<double>(logp[i]);
+        const float v = row[a];
+        acc[a] += static_cast<double>(expf(v));
+        if (v > best) {
+          best = v;
+          arg = a;
+        }
       }
     }
-    red[t] = acc;
-    redi[t] = cnt;
-    __syncthreads();
-    for (int o = blockDim.x >> 1; o > 0; o >>= 1) {
-      if (t < o) {
-        red[t] += red[t + o];
-        redi[t] += redi[t + o];
-      }
-      __syncthreads();
+#pragma unroll
+    for (int a = 0; a < CPMTP_MAX_R; ++a) cnt[a] += (a == arg) ? 1 : 0;
+    acc[CPMTP_MAX_R] += static_cast<double>(logp[i]);
+  }
+#pragma unroll
+  for (int a = 0; a <= CPMTP_MAX_R; ++a) {
+    if (a < r || a == CPMTP_MAX_R) {
+      double v = acc[a];
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+      if (lane == 0) sum_s[warp][a] = v;
     }
-    if (t == 0) {
-      if (a < r) {
-        wbar_s[a] = red[0] / N;
-        if (wbar != nullptr) wbar[a] = static_cast<float>(wbar_s[a]);
-        if (counts != nullptr) counts[a] = redi[0];
-      } else if (loss != nullptr) {
-        double aux = 0.0;
-        for (int b = 0; b < r; ++b) aux += wbar_s[b] * wbar_s[b];
-        *loss = static_cast<float>(-red[0] / N + static_cast<double>(aux_coef) * aux);
-      }
+  }
+#pragma unroll
+  for (int a = 0; a < CPMTP_MAX_R; ++a) {
+    if (a < r) {
+      int c = cnt[a];
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) c += __shfl_xor_sync(0xffffffffu, c, o);
+      if (lane == 0) cnt_s[warp][a] = c;
     }
-    __syncthreads();
+  }
+  __syncthreads();
+  if (t <= CPMTP_MAX_R && (t < r || t == CPMTP_MAX_R)) {
+    double v = 0.0;
+    int c = 0;
+    for (int w = 0; w < nwarps; ++w) {
+      v += sum_s[w][t];
+      if (t < r) c += cnt_s[w][t];
+    }
+    sum_s[0][t] = v;
+    if (t < r) {
+      if (wbar != nullptr) wbar[t] = static_cast<float>(v / N);
+      if (counts != nullptr) counts[t] = c;
+    }
+  }
+  __syncthreads();
+  if (t == 0 && loss != nullptr) {
+    double aux = 0.0;
+    for (int b2 = 0; b2 < r; ++b2) aux += (sum_s[0][b2] / N) * (sum_s[0][b2] / N);
+    *loss = static_cast<float>(-sum_s[0][CPMTP_MAX_R] / N + static_cast<double>(aux_coef) * aux);
   }
 }
 
