@@ -44,8 +44,8 @@ WORKLOADS = {
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel, from the ncu
 # captures summarised under profiles/ (None until captured, or once the kernel has changed since).
 NCU_TRAFFIC_BYTES = {
-    "train_fwd": 1.215086e9 + 5.97632e6,   # profiles/lse_train_fwd.md
-    "decode_1": 1.051697e9 + 3.96288e6,    # profiles/decode_1.md
+    "train_fwd": 1.236112e9 + 5.9648e6,   # profiles/lse_train_fwd.md
+    "decode_1": 1.05168e9 + 3.763968e6,    # profiles/decode_1.md
 }
 
 
@@ -69,7 +69,7 @@ class ClockSampler:
         try:
             self.proc = subprocess.Popen(
                 ["nvidia-smi", f"--id={gpu_index}", f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits",
-                 "-lms", "100"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+                 "-lms", "50"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
         except OSError:
             self.proc = None
 
