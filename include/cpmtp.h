@@ -28,6 +28,14 @@
  *    expired (results invalid).
  *  - Limits: d % 64 == 0, 1 <= r <= 32, 1 <= n <= 8, N >= 1, V >= 2,
  *    N*n*r*d < 2^40.
+ *  - Threads: calls may be made from several host threads as long as each uses
+ *    its own stream, workspace and outputs; the per-stage profiling calls are
+ *    the exception (one thread, one device).
+ *  - Environment knobs, read at call time, for testing and tuning only:
+ *    CPMTP_BWD_CHUNK_ROWS / CPMTP_BWD_CHUNK_HEADS (rows / heads of logit gradients
+ *    recomputed at a time in the backward passes; also changes the workspace the
+ *    backward needs, so set it before querying cpmtp_workspace_bytes),
+ *    CPMTP_LSE_GROUP_MB and CPMTP_LSE_SPLITS (schedule of the fused unembedding).
  */
 #ifndef CPMTP_H
 #define CPMTP_H
