@@ -31,6 +31,8 @@ WORKLOADS = {
     "train_fwd": ("train_fwd", "fwd", {}, None),
     "train_fwd_bwd": ("train_fwd_bwd", "fwd_bwd", {}, None),
     "bigvocab_fwd_bwd": ("bigvocab_fwd_bwd", "fwd_bwd", {"targets": "zipf"}, 1.0),
+    # head-only fine-tuning as in the paper: shared unembedding and trunk frozen (no dE, no dh)
+    "finetune_fwd_bwd": ("train_fwd_bwd", "fwd_bwd", {}, None),
     "decode_1": ("decode_1", "score", {}, None),
     "decode_8": ("decode_8", "score", {}, None),
     "decode_64": ("decode_64", "score", {}, None),
@@ -206,6 +208,7 @@ def run_ours(args, rank: int, world: int, local_rank: int):
     ws_bwd = binding.alloc_workspace(binding.workspace_bytes(cs, binding.OP_BACKWARD)) if kind == "fwd_bwd" else None
     ws_smp = binding.alloc_workspace(binding.workspace_bytes(cs, binding.OP_SAMPLE)) if kind == "sample" else None
     out_f, out_b, out_s = {}, {}, {}
+    skip = ("dE", "dh") if args.workload == "finetune_fwd_bwd" else ()
 
     def step():
         if kind == "fwd":
@@ -214,7 +217,7 @@ def run_ours(args, rank: int, world: int, local_rank: int):
             binding.forward(h, W_head, E, W_g, x, aux_coef=aux, saved=saved, workspace=ws_fwd, dev_status=status,
                             out=out_f)
             binding.backward(h, W_head, E, W_g, x, saved, aux_coef=aux, workspace=ws_bwd, dev_status=status,
-                             out=out_b)
+                             out=out_b, skip=skip)
         elif kind == "sample":
             binding.sample_draft(h, W_head, E, W_g, shape.n, topk=5, workspace=ws_smp, dev_status=status, out=out_s)
         elif kind == "full_fwd_bwd":
@@ -247,7 +250,7 @@ def run_ours(args, rank: int, world: int, local_rank: int):
                              workspace=ws_fwd, dev_status=status)
         if kind == "fwd_bwd":
             binding.backward(h, W_head, E, W_g, x, saved, aux_coef=aux, workspace=ws_bwd, dev_status=status,
-                             out=out_b)
+                             out=out_b, skip=skip)
         torch.cuda.current_stream().synchronize()   # the step's result is read on the host
 
     def barrier():

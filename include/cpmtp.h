@@ -126,7 +126,11 @@ int cpmtp_forward(const cpmtp_shape* shape, const void* h, const void* W_head, c
  * log-likelihood that training minimises).  The logits are recomputed tile by
  * tile from `saved` (as filled by cpmtp_forward on the same inputs).  Outputs are
  * bf16, rounded once from fp32 accumulators:
- *   dh [N,d], dW_head [n*r,d,d], dE [V,d], dW_g [r,d]; all required.
+ *   dh [N,d], dW_head [n*r,d,d], dE [V,d], dW_g [r,d].
+ * Any of the four may be NULL and is then not computed (at least one must be
+ * given): with the shared unembedding frozen, as in the paper's fine-tuning
+ * set-up, dE = NULL skips a quarter of the backward work; with a frozen trunk
+ * dh = NULL skips its GEMM.
  */
 int cpmtp_backward(const cpmtp_shape* shape, const void* h, const void* W_head, const void* E,
                    const void* W_g, const int32_t* x, const cpmtp_saved* saved,

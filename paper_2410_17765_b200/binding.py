@@ -210,20 +210,22 @@ def forward(h, W_head, E, W_g, x, *, aux_coef: Optional[float] = None, saved: Op
 
 def backward(h, W_head, E, W_g, x, saved: Saved, *, aux_coef: Optional[float] = None,
              dloss_dlogp: Optional[torch.Tensor] = None, workspace: Optional[torch.Tensor] = None,
-             dev_status: Optional[torch.Tensor] = None, out: Optional[dict] = None) -> dict:
-    """cpmtp_backward on device tensors; returns {"dh", "dW_head", "dE", "dW_g"} (bf16 device tensors)."""
+             dev_status: Optional[torch.Tensor] = None, out: Optional[dict] = None,
+             skip: tuple = ()) -> dict:
+    """cpmtp_backward on device tensors; returns {"dh", "dW_head", "dE", "dW_g"} (bf16 device tensors).
+    Names listed in `skip` are not computed (passed as NULL)."""
     lib = load_library()
     shape = _shape_of(h, W_head, E, W_g, x, aux_coef)
     if workspace is None:
         workspace = alloc_workspace(workspace_bytes(shape, OP_BACKWARD), h.device)
     res = out if out is not None else {}
     for name, ref in (("dh", h), ("dW_head", W_head), ("dE", E), ("dW_g", W_g)):
-        if name not in res:
+        if name not in res and name not in skip:
             res[name] = torch.empty_like(ref)
     cs = saved.c_struct()
     rc = lib.cpmtp_backward(ctypes.byref(shape), _ptr(h), _ptr(W_head), _ptr(E), _ptr(W_g), _ptr(x),
-                            ctypes.byref(cs), _ptr(dloss_dlogp), _ptr(res["dh"]), _ptr(res["dW_head"]),
-                            _ptr(res["dE"]), _ptr(res["dW_g"]), _ptr(workspace), workspace.numel(),
+                            ctypes.byref(cs), _ptr(dloss_dlogp), _ptr(res.get("dh")), _ptr(res.get("dW_head")),
+                            _ptr(res.get("dE")), _ptr(res.get("dW_g")), _ptr(workspace), workspace.numel(),
                             _ptr(dev_status), _stream())
     _check(rc)
     return res

@@ -820,10 +820,12 @@ int cpmtp_backward(const cpmtp_shape* shape, const void* h, const void* W_head, 
   DeviceInfo* di = nullptr;
   const int rc = check_common(shape, h, W_head, E, W_g, x, workspace, &di);
   if (rc != CPMTP_OK) return rc;
-  if (saved == nullptr || !dh || !dW_head || !dE || !dW_g) return CPMTP_ERR_NULL;
+  if (saved == nullptr) return CPMTP_ERR_NULL;
+  if (!dh && !dW_head && !dE && !dW_g) return CPMTP_ERR_NULL;   // nothing asked for
   const int rs = check_saved(saved);
   if (rs != CPMTP_OK) return rs;
   if (!aligned(dh, 16) || !aligned(dW_head, 16) || !aligned(dE, 16) || !aligned(dW_g, 16)) return CPMTP_ERR_ALIGN;
+  const bool need_dz = dh != nullptr || dW_head != nullptr;   // dz feeds only these two
   const cpmtp_shape& s = *shape;
   const BwdLayout L = bwd_layout(s);
   if (workspace_bytes < L.total) return CPMTP_ERR_WORKSPACE;
@@ -856,19 +858,19 @@ int cpmtp_backward(const cpmtp_shape* shape, const void* h, const void* W_head, 
     const uint16_t* zc = z + row0 * d;
     const int m_tiles = (rows + kBM - 1) / kBM;
     // recompute logits tile by tile -> G = dloss/dS (bf16), never more than one chunk
-    {
+    if (need_dz || dE != nullptr) {
       ProfScope prof(CPMTP_STAGE_LOGIT_GRAD, st);
       EpiLogitGrad<kBN>::Params ep{G, saved->lse, coef, x, row0, rows, L.ldg, V, K, s.n, s.r};
       CPMTP_TRY((gemm_auto<false, false, EpiLogitGrad<kBN>>(zc, d, Eb, d, rows, V, d, 2048, ep, dev_status, sms, st)));
     }
     // dz[rows, d] = G[rows, V] * E[V, d]
-    {
+    if (need_dz) {
       ProfScope prof(CPMTP_STAGE_DZ, st);
       EpiStoreBf16<kBN, false>::Params ep{dz + row0 * d, nullptr, nullptr, rows, d, d, 0};
       CPMTP_TRY((gemm_auto<false, true, EpiStoreBf16<kBN, false>>(G, L.ldg, Eb, d, rows, d, V, 2048, ep, dev_status, sms, st)));
     }
     // dE[V, d] (+)= G^T[V, rows] * z[rows, d]
-    {
+    if (dE != nullptr) {
       ProfScope prof(CPMTP_STAGE_DE, st);
       if (L.chunks == 1) {
         EpiStoreBf16<kBN, false>::Params ep{static_cast<uint16_t*>(dE), nullptr, nullptr, V, d, d, 0};
@@ -879,25 +881,25 @@ int cpmtp_backward(const cpmtp_shape* shape, const void* h, const void* W_head, 
       }
     }
   }
-  if (L.chunks > 1) {
+  if (L.chunks > 1 && dE != nullptr) {
     ProfScope prof(CPMTP_STAGE_DE_CONVERT, st);
     f32_to_bf16_kernel<<<sms * 8, 256, 0, st>>>(dE32, static_cast<uint16_t*>(dE), static_cast<size_t>(V) * d);
     CPMTP_TRY(cudaGetLastError());
   }
   // dW_head[K*d, d] = dz^T[K*d, N] * h[N, d]
-  {
+  if (dW_head != nullptr) {
     ProfScope prof(CPMTP_STAGE_DW_HEAD, st);
     EpiStoreBf16<kBN, false>::Params ep{static_cast<uint16_t*>(dW_head), nullptr, nullptr, ncols, d, d, 0};
     CPMTP_TRY((gemm_auto<true, true, EpiStoreBf16<kBN, false>>(dz, ncols, h, d, ncols, d, s.N, 2048, ep, dev_status, sms, st)));
   }
   // dh[N, d] = dz[N, K*d] * W_cat[K*d, d] + dg * W_g
-  {
+  if (dh != nullptr) {
     ProfScope prof(CPMTP_STAGE_DH, st);
     EpiStoreBf16<kBN, true>::Params ep{static_cast<uint16_t*>(dh), dg, static_cast<const uint16_t*>(W_g), s.N, d, d, s.r};
     CPMTP_TRY((gemm_auto<false, true, EpiStoreBf16<kBN, true>>(dz, ncols, W_head, d, s.N, d, ncols, 2048, ep, dev_status, sms, st)));
   }
   // dW_g[r, d] = dg^T * h
-  {
+  if (dW_g != nullptr) {
     ProfScope prof(CPMTP_STAGE_DW_G, st);
     dim3 grid((d + 127) / 128, L.dwg_slices);
     dwg_partial_kernel<CPMTP_MAX_R><<<grid, 128, 0, st>>>(dg, static_cast<const uint16_t*>(h), dwg_part, s.N, d, s.r,

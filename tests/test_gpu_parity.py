@@ -190,3 +190,24 @@ def test_forward_host_matches_device_forward():
     torch.cuda.synchronize()
     assert torch.equal(logp_host, want["logp"].cpu())
     assert torch.equal(loss_host, want["loss"].cpu())
+
+
+@pytest.mark.parametrize("skip", [("dE",), ("dh",), ("dE", "dh", "dW_g"), ("dh", "dW_head"), ("dW_head", "dE", "dW_g")])
+def test_backward_skips_outputs_that_are_not_asked_for(skip):
+    from paper_2410_17765_b200 import binding
+
+    shape = CASES["wide"]["shape"]
+    inp = synth.make_inputs(shape, seed=0)
+    dev = to_dev(inp)
+    saved = binding.Saved.alloc(binding.make_shape(shape.N, shape.d, shape.V, shape.n, shape.r))
+    binding.forward(*dev, saved=saved)
+    full = binding.backward(*dev, saved)
+    part = binding.backward(*dev, saved, skip=skip)
+    torch.cuda.synchronize()
+    for key in ("dh", "dW_head", "dE", "dW_g"):
+        if key in skip:
+            assert key not in part
+        else:
+            assert torch.equal(part[key], full[key]), key
+    with pytest.raises(binding.CpmtpError):
+        binding.backward(*dev, saved, skip=("dh", "dW_head", "dE", "dW_g"))
