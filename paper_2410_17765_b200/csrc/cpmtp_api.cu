@@ -851,12 +851,10 @@ int cpmtp_backward(const cpmtp_shape* shape, const void* h, const void* W_head, 
     CPMTP_TRY(cudaGetLastError());
   }
 
-  const int d_tiles = (d + kBN - 1) / kBN;
   for (int c = 0; c < L.chunks; ++c) {
     const long long row0 = static_cast<long long>(c) * L.chunk_rows;
     const int rows = static_cast<int>((L.M - row0) < L.chunk_rows ? (L.M - row0) : L.chunk_rows);
     const uint16_t* zc = z + row0 * d;
-    const int m_tiles = (rows + kBM - 1) / kBM;
     // recompute logits tile by tile -> G = dloss/dS (bf16), never more than one chunk
     if (need_dz || dE != nullptr) {
       ProfScope prof(CPMTP_STAGE_LOGIT_GRAD, st);
