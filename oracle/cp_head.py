@@ -155,10 +155,37 @@ class Gradients:
     c: np.ndarray        # [N, r]  gradient w.r.t. every C[i, s, alpha] (same for all s)
 
 
+def _coefficients(fw: Forward, N: int, aux_coef: float, dloss_dlogp, dloss_dprefix):
+    """Gradient of the objective w.r.t. every C[i, s, alpha] (returned as c3 [N, n, r]) and w.r.t. the
+    gate logits (dg [N, r]).
+
+    Plain objective  sum_i up_i logp_i:  c3[i, s, :] = up_i q[i, :] for every s.
+    Per-token objective  sum_i sum_s up[i, s] * prefix[i, s]  with prefix[i, s] = log P(x_1..x_{s+1}), e.g. the
+    discounted cross-entropy part of the fine-tuning loss (Eq. 14 and the sum after it: CE_k = prefix_{k-1} -
+    prefix_k):  prefix_s depends on C[t, :] for t <= s through its own expert posterior q_s, hence
+      c3[i, t, :] = sum_{s >= t} up[i, s] q_s[i, :],   dg = sum_s up[i, s] (q_s - w)."""
+    w = np.exp(fw.logw)
+    u = 2.0 * aux_coef * fw.wbar / N
+    aux_dg = w * (u[None, :] - (w @ u)[:, None])
+    n = fw.C.shape[1]
+    if dloss_dprefix is None:
+        up = np.full(N, -1.0 / N) if dloss_dlogp is None else _f64(dloss_dlogp)
+        c = up[:, None] * fw.q
+        return np.repeat(c[:, None, :], n, axis=1), up[:, None] * (fw.q - w) + aux_dg
+    ups = _f64(dloss_dprefix)                                   # [N, n]
+    a_s = fw.logw[:, None, :] + np.cumsum(fw.C, axis=1)         # [N, n, r]
+    q_s = np.exp(a_s - logsumexp(a_s, axis=2)[:, :, None])
+    weighted = ups[:, :, None] * q_s
+    c3 = np.cumsum(weighted[:, ::-1, :], axis=1)[:, ::-1, :]    # suffix sums over s
+    dg = (weighted - ups[:, :, None] * w[:, None, :]).sum(axis=1) + aux_dg
+    return c3, dg
+
+
 def backward(h, W_head, E, W_g, x, n: int, r: int, *, aux_coef: float = 0.0,
-             dloss_dlogp=None) -> Gradients:
+             dloss_dlogp=None, dloss_dprefix=None) -> Gradients:
     """Gradient of  loss = sum_i up_i * logp_i + aux_coef * sum_alpha wbar_alpha^2
-    with up_i = dloss_dlogp[i] (default -1/N, the mean negative log-likelihood).
+    with up_i = dloss_dlogp[i] (default -1/N, the mean negative log-likelihood); or, with
+    dloss_dprefix [N, n], of  sum_i sum_s dloss_dprefix[i, s] * log P(x_1..x_{s+1})  (see _coefficients).
 
     Chain rule through Eq. 9, Eq. 8 and Eq. 7:
       d loss / d a[i, alpha]      = up_i * q[i, alpha]            (softmax of the outer logsumexp)
@@ -175,11 +202,8 @@ def backward(h, W_head, E, W_g, x, n: int, r: int, *, aux_coef: float = 0.0,
     V = Ed.shape[0]
     K = n * r
     fw = forward(h, W_head, E, W_g, x, n, r, aux_coef=aux_coef)
-    up = np.full(N, -1.0 / N) if dloss_dlogp is None else _f64(dloss_dlogp)
-    c = up[:, None] * fw.q
-    w = np.exp(fw.logw)
-    u = 2.0 * aux_coef * fw.wbar / N
-    dg = up[:, None] * (fw.q - w) + w * (u[None, :] - (w @ u)[:, None])
+    c3, dg = _coefficients(fw, N, aux_coef, dloss_dlogp, dloss_dprefix)
+    c = c3[:, -1, :] if dloss_dprefix is None else c3
 
     dh = dg @ Wg
     dW_g = dg.T @ hd
@@ -192,8 +216,8 @@ def backward(h, W_head, E, W_g, x, n: int, r: int, *, aux_coef: float = 0.0,
         z = hd @ Wk.T
         S = z @ Ed.T
         P = np.exp(S - fw.lse[:, k][:, None])
-        G = -c[:, alpha][:, None] * P
-        G[rows, xi[:, s]] += c[:, alpha]
+        G = -c3[:, s, alpha][:, None] * P
+        G[rows, xi[:, s]] += c3[:, s, alpha]
         dz = G @ Ed
         dE += G.T @ z
         dW_head[k] = dz.T @ hd
@@ -302,18 +326,15 @@ class GradientsFull:
     dW_g: np.ndarray     # [r, d]
 
 
-def backward_full(h, W_full, W_g, x, n: int, r: int, *, aux_coef: float = 0.0, dloss_dlogp=None) -> GradientsFull:
+def backward_full(h, W_full, W_g, x, n: int, r: int, *, aux_coef: float = 0.0, dloss_dlogp=None,
+                  dloss_dprefix=None) -> GradientsFull:
     """Gradient of the same objective as `backward`, for the full head:
     dS as there; dW_full[k] = dS[:, k, :]^T h, dh = sum_k dS[:, k, :] W_full[k] + dg W_g."""
     hd, Wg, xi = _f64(h), _f64(W_g), _i64(x)
     N, d = hd.shape
     K = n * r
     fw = forward_full(h, W_full, W_g, x, n, r, aux_coef=aux_coef)
-    up = np.full(N, -1.0 / N) if dloss_dlogp is None else _f64(dloss_dlogp)
-    c = up[:, None] * fw.q
-    w = np.exp(fw.logw)
-    u = 2.0 * aux_coef * fw.wbar / N
-    dg = up[:, None] * (fw.q - w) + w * (u[None, :] - (w @ u)[:, None])
+    c3, dg = _coefficients(fw, N, aux_coef, dloss_dlogp, dloss_dprefix)
     dh = dg @ Wg
     dW_g = dg.T @ hd
     V = _f64(W_full[0]).shape[0]
@@ -323,8 +344,8 @@ def backward_full(h, W_full, W_g, x, n: int, r: int, *, aux_coef: float = 0.0, d
         s, alpha = divmod(k, r)
         Wk = _f64(W_full[k])
         S = hd @ Wk.T
-        G = -c[:, alpha][:, None] * np.exp(S - fw.lse[:, k][:, None])
-        G[rows, xi[:, s]] += c[:, alpha]
+        G = -c3[:, s, alpha][:, None] * np.exp(S - fw.lse[:, k][:, None])
+        G[rows, xi[:, s]] += c3[:, s, alpha]
         dW_full[k] = G.T @ hd
         dh += G @ Wk
     return GradientsFull(dh=dh, dW_full=dW_full, dW_g=dW_g)

@@ -94,3 +94,45 @@ def test_gradients_are_additive_over_position_chunks():
         acc += part.dE
         assert np.allclose(part.dh, full.dh[lo:hi], atol=1e-15)
     assert np.allclose(acc, full.dE, atol=1e-15)
+
+
+def test_per_token_objective_gradients_match_finite_differences():
+    # objective sum_i sum_s up[i, s] * log P(x_1..x_{s+1}) + aux: e.g. a discounted per-token cross-entropy
+    p, s = problem(seed=11, N=3, n=3, r=2)
+    rng = np.random.default_rng(3)
+    ups = rng.normal(size=(s.N, s.n))
+    aux = 0.8
+
+    def f():
+        fw = cp_head.forward(p["h"], p["W_head"], p["E"], p["W_g"], p["x"], s.n, s.r, aux_coef=aux)
+        return float(np.sum(ups * cp_head.prefix_log_probs(fw)) + aux * np.sum(fw.wbar ** 2))
+
+    g = cp_head.backward(p["h"], p["W_head"], p["E"], p["W_g"], p["x"], s.n, s.r, aux_coef=aux, dloss_dprefix=ups)
+    for name, grad in [("h", g.dh), ("W_head", g.dW_head), ("E", g.dE), ("W_g", g.dW_g)]:
+        arr = p[name]
+        for fi in rng.choice(arr.size, size=min(arr.size, 20), replace=False):
+            idx = np.unravel_index(fi, arr.shape)
+            old = arr[idx]
+            arr[idx] = old + 1e-6
+            fp = f()
+            arr[idx] = old - 1e-6
+            fm = f()
+            arr[idx] = old
+            assert abs((fp - fm) / 2e-6 - grad[idx]) <= 1e-6 * max(1.0, abs(grad[idx])) + 1e-8, (name, idx)
+    # weights on the last prefix only reproduce the plain objective
+    last = np.zeros((s.N, s.n))
+    last[:, -1] = -1.0 / s.N
+    a = cp_head.backward(p["h"], p["W_head"], p["E"], p["W_g"], p["x"], s.n, s.r, dloss_dprefix=last)
+    b = cp_head.backward(p["h"], p["W_head"], p["E"], p["W_g"], p["x"], s.n, s.r)
+    assert np.allclose(a.dE, b.dE, atol=1e-15) and np.allclose(a.dh, b.dh, atol=1e-15)
+    # discounted cross-entropy: sum_k gamma^k CE_k with CE_k = prefix_{k-1} - prefix_k is such a weighting
+    gamma = 0.7
+    wts = np.zeros((s.N, s.n))
+    for k in range(s.n):
+        wts[:, k] -= gamma ** k / s.N
+        if k > 0:
+            wts[:, k - 1] += gamma ** k / s.N
+    fw = cp_head.forward(p["h"], p["W_head"], p["E"], p["W_g"], p["x"], s.n, s.r)
+    pre = cp_head.prefix_log_probs(fw)
+    ce = -np.diff(pre, axis=1, prepend=0.0)                      # CE_k = -log p(x_k | x_<k)
+    assert abs(np.sum(wts * pre) - np.sum((gamma ** np.arange(s.n))[None, :] * ce) / s.N) < 1e-12
