@@ -72,6 +72,10 @@ enum {
 
 /* flags */
 #define CPMTP_FLAG_AUX 1u /* add aux_coef * sum_a wbar_a^2 to the loss (soft form of Eq. 10) */
+/* Backward only: `dloss_dlogp` is [N, n] and weighs the PREFIX log-probabilities, the objective being
+ * sum_i sum_s dloss_dlogp[i, s] * log P(x[i, 0..s]).  The discounted per-token cross-entropy of the
+ * fine-tuning loss (Eq. 14 and the sum after it, CE_k = log P(x[0..k-1]) - log P(x[0..k])) is of this form. */
+#define CPMTP_FLAG_PER_TOKEN 2u
 
 typedef struct cpmtp_shape {
   int32_t N;        /* positions */

@@ -17,6 +17,7 @@ from .build import LIB_PATH
 
 OP_FORWARD, OP_BACKWARD, OP_SCORE, OP_SAMPLE, OP_FORWARD_FULL, OP_BACKWARD_FULL = 0, 1, 2, 3, 4, 5
 FLAG_AUX = 1
+FLAG_PER_TOKEN = 2
 
 EXPORTS = [
     "cpmtp_version", "cpmtp_status_string", "cpmtp_workspace_bytes", "cpmtp_forward", "cpmtp_backward",
@@ -211,11 +212,16 @@ def forward(h, W_head, E, W_g, x, *, aux_coef: Optional[float] = None, saved: Op
 def backward(h, W_head, E, W_g, x, saved: Saved, *, aux_coef: Optional[float] = None,
              dloss_dlogp: Optional[torch.Tensor] = None, workspace: Optional[torch.Tensor] = None,
              dev_status: Optional[torch.Tensor] = None, out: Optional[dict] = None,
-             skip: tuple = ()) -> dict:
+             skip: tuple = (), dloss_dprefix: Optional[torch.Tensor] = None) -> dict:
     """cpmtp_backward on device tensors; returns {"dh", "dW_head", "dE", "dW_g"} (bf16 device tensors).
-    Names listed in `skip` are not computed (passed as NULL)."""
+    Names listed in `skip` are not computed (passed as NULL).  dloss_dprefix [N, n] fp32 selects the
+    per-token objective sum_i sum_s dloss_dprefix[i, s] * log P(x[i, 0..s]) (CPMTP_FLAG_PER_TOKEN)."""
     lib = load_library()
     shape = _shape_of(h, W_head, E, W_g, x, aux_coef)
+    if dloss_dprefix is not None:
+        assert dloss_dlogp is None and dloss_dprefix.shape == (shape.N, shape.n) and dloss_dprefix.dtype == torch.float32
+        shape.flags |= FLAG_PER_TOKEN
+        dloss_dlogp = dloss_dprefix.contiguous()
     if workspace is None:
         workspace = alloc_workspace(workspace_bytes(shape, OP_BACKWARD), h.device)
     res = out if out is not None else {}
@@ -318,10 +324,16 @@ def forward_full(h, W_full, W_g, x, *, aux_coef: Optional[float] = None, saved: 
 
 def backward_full(h, W_full, W_g, x, saved: Saved, *, aux_coef: Optional[float] = None,
                   dloss_dlogp: Optional[torch.Tensor] = None, workspace: Optional[torch.Tensor] = None,
-                  dev_status: Optional[torch.Tensor] = None, out: Optional[dict] = None) -> dict:
-    """cpmtp_backward_full; returns {"dh", "dW_full", "dW_g"} (bf16 device tensors)."""
+                  dev_status: Optional[torch.Tensor] = None, out: Optional[dict] = None,
+                  dloss_dprefix: Optional[torch.Tensor] = None) -> dict:
+    """cpmtp_backward_full; returns {"dh", "dW_full", "dW_g"} (bf16 device tensors).
+    dloss_dprefix as for backward()."""
     lib = load_library()
     shape = _shape_full(h, W_full, W_g, x, aux_coef)
+    if dloss_dprefix is not None:
+        assert dloss_dlogp is None and dloss_dprefix.shape == (shape.N, shape.n) and dloss_dprefix.dtype == torch.float32
+        shape.flags |= FLAG_PER_TOKEN
+        dloss_dlogp = dloss_dprefix.contiguous()
     if workspace is None:
         workspace = alloc_workspace(workspace_bytes(shape, OP_BACKWARD_FULL), h.device)
     res = out if out is not None else {}

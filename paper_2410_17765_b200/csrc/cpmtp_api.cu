@@ -172,7 +172,7 @@ BwdLayout bwd_layout(const cpmtp_shape& s) {
   L.dwg_slices = (s.N + L.dwg_rows_per_slice - 1) / L.dwg_rows_per_slice;
   size_t off = 0;
   auto take = [&](size_t bytes) { size_t o = off; off = align_up(off + bytes); return o; };
-  L.coef = take(sizeof(float) * s.N * s.r);
+  L.coef = take(sizeof(float) * static_cast<size_t>(s.N) * L.K);
   L.dg = take(sizeof(float) * s.N * s.r);
   L.dz = take(2ull * L.M * s.d);
   L.G = take(2ull * L.chunk_rows * L.ldg);
@@ -263,7 +263,7 @@ FullBwdLayout full_bwd_layout(const cpmtp_shape& s) {
   L.dwg_slices = (s.N + L.dwg_rows_per_slice - 1) / L.dwg_rows_per_slice;
   size_t off = 0;
   auto take = [&](size_t bytes) { size_t o = off; off = align_up(off + bytes); return o; };
-  L.coef = take(sizeof(float) * s.N * s.r);
+  L.coef = take(sizeof(float) * static_cast<size_t>(s.N) * L.K);
   L.dg = take(sizeof(float) * s.N * s.r);
   L.G = take(2ull * s.N * L.heads_per_chunk * L.ldv);
   L.dh32 = take(sizeof(float) * static_cast<size_t>(s.N) * s.d);
@@ -687,10 +687,12 @@ int cpmtp_backward_full(const cpmtp_shape* shape, const void* h, const void* W_f
   const int sms = di->sms;
   const int K = L.K, d = s.d, V = s.V;
   const float aux = (s.flags & CPMTP_FLAG_AUX) ? s.aux_coef : 0.f;
+  const int per_token = (s.flags & CPMTP_FLAG_PER_TOKEN) ? 1 : 0;
+  if (per_token && (dloss_dlogp == nullptr || saved->tgt == nullptr)) return CPMTP_ERR_NULL;
   {
     ProfScope prof(CPMTP_STAGE_COEFF, st);
-    coeff_kernel<<<(s.N + 255) / 256, 256, 0, st>>>(saved->q, saved->logw, saved->wbar, dloss_dlogp, coef, dg, s.N,
-                                                   s.r, aux);
+    coeff_kernel<<<(s.N + 127) / 128, 128, 0, st>>>(saved->q, saved->logw, saved->wbar, saved->lse, saved->tgt,
+                                                   dloss_dlogp, per_token, coef, dg, s.N, s.n, s.r, aux);
     CPMTP_TRY(cudaGetLastError());
   }
   const bool wide = use_wide(s.N, d);
@@ -843,11 +845,13 @@ int cpmtp_backward(const cpmtp_shape* shape, const void* h, const void* W_head, 
   const int K = L.K, d = s.d, V = s.V;
   const int ncols = K * d;
   const float aux = (s.flags & CPMTP_FLAG_AUX) ? s.aux_coef : 0.f;
+  const int per_token = (s.flags & CPMTP_FLAG_PER_TOKEN) ? 1 : 0;
+  if (per_token && dloss_dlogp == nullptr) return CPMTP_ERR_NULL;
 
   {
     ProfScope prof(CPMTP_STAGE_COEFF, st);
-    coeff_kernel<<<(s.N + 255) / 256, 256, 0, st>>>(saved->q, saved->logw, saved->wbar, dloss_dlogp, coef, dg,
-                                                   s.N, s.r, aux);
+    coeff_kernel<<<(s.N + 127) / 128, 128, 0, st>>>(saved->q, saved->logw, saved->wbar, saved->lse, saved->tgt,
+                                                   dloss_dlogp, per_token, coef, dg, s.N, s.n, s.r, aux);
     CPMTP_TRY(cudaGetLastError());
   }
 

@@ -269,7 +269,7 @@ struct EpiLogitGrad {
   struct Params {
     uint16_t* G;          // [rows, ldg] bf16
     const float* lse;     // [N*K]
-    const float* coef;    // [N, r]
+    const float* coef;    // [N, K]  d objective / d C per head
     const int32_t* x;     // [N, n]
     long long row0;
     int rows, ldg, V, K, n, r;
@@ -286,7 +286,7 @@ struct EpiLogitGrad {
       const long long i = grow / p.K;
       const int k = static_cast<int>(grow - i * p.K);
       st.lse2 = p.lse[grow] * kLog2e;
-      st.coef = p.coef[i * p.r + (k % p.r)];
+      st.coef = p.coef[grow];
       const int tok = p.x[i * p.n + k / p.r];
       st.tok = tok < 0 ? 0 : (tok >= p.V ? p.V - 1 : tok);
     }
@@ -331,7 +331,7 @@ struct EpiLogitGradFull {
   struct Params {
     uint16_t* G;          // [M, ldg] bf16, ldg = heads * ldv
     const float* lse;     // [M, K]
-    const float* coef;    // [M, r]
+    const float* coef;    // [M, K]  d objective / d C per head
     const int32_t* x;     // [M, n]
     int M, V, K, n, r, tph, ldv, ldg, k0;
   };
@@ -353,7 +353,7 @@ struct EpiLogitGradFull {
       st.tok = -1;
       if (valid) {
         st.lse2 = p.lse[static_cast<size_t>(row) * p.K + k] * kLog2e;
-        st.coef = p.coef[static_cast<size_t>(row) * p.r + (k % p.r)];
+        st.coef = p.coef[static_cast<size_t>(row) * p.K + k];
         const int tok = p.x[static_cast<size_t>(row) * p.n + k / p.r];
         st.tok = tok < 0 ? 0 : (tok >= p.V ? p.V - 1 : tok);
       }

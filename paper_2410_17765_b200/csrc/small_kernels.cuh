@@ -190,24 +190,70 @@ __global__ void __launch_bounds__(kFinalizeThreads) finalize_kernel(const float*
   }
 }
 
-// Backward coefficients (derivative of Eq. 9 and of the gate softmax of Eq. 7).
-//   c[i,a]  = up_i * q[i,a]
-//   dg[i,b] = up_i * (q[i,b] - w[i,b]) + w[i,b] * (u_b - sum_g w[i,g] u_g),  u_b = 2 aux wbar_b / N
+// Backward coefficients (derivative of Eq. 9 and of the gate softmax of Eq. 7), one thread per position.
+//   coef[i, t*r + a] = d objective / d C[i, t, a]        dg[i, b] = d objective / d (W_g h)[i, b]
+// Plain objective  sum_i up_i logp_i  (up == nullptr: up_i = -1/N):
+//   coef[i, t, a] = up_i q[i, a] for every t;  dg = up_i (q - w) + aux part.
+// Per-token objective  sum_i sum_s up[i, s] * log P(x_1..x_{s+1})  (per_token != 0, up is [N, n]):
+//   with q_s the expert posterior after s+1 tokens,  coef[i, t, a] = sum_{s >= t} up[i, s] q_s[i, a],
+//   dg = sum_s up[i, s] (q_s - w) + aux part.
+// aux part (soft balance term): w_b (u_b - sum_g w_g u_g), u_b = 2 aux wbar_b / N.
 __global__ void coeff_kernel(const float* __restrict__ q, const float* __restrict__ logw,
-                             const float* __restrict__ wbar, const float* __restrict__ up,
-                             float* __restrict__ coef, float* __restrict__ dg, int N, int r,
+                             const float* __restrict__ wbar, const float* __restrict__ lse,
+                             const float* __restrict__ tgt, const float* __restrict__ up, int per_token,
+                             float* __restrict__ coef, float* __restrict__ dg, int N, int n, int r,
                              float aux_coef) {
   const int i = blockIdx.x * blockDim.x + threadIdx.x;
   if (i >= N) return;
-  const float u_i = up != nullptr ? up[i] : -1.0f / N;
+  const int K = n * r;
   const float scale = 2.0f * aux_coef / N;
   float wu = 0.f;
   for (int b = 0; b < r; ++b) wu += expf(logw[static_cast<size_t>(i) * r + b]) * scale * wbar[b];
+  if (!per_token) {
+    const float u_i = up != nullptr ? up[i] : -1.0f / N;
+    for (int b = 0; b < r; ++b) {
+      const float w = expf(logw[static_cast<size_t>(i) * r + b]);
+      const float qq = q[static_cast<size_t>(i) * r + b];
+      for (int t = 0; t < n; ++t) coef[static_cast<size_t>(i) * K + t * r + b] = u_i * qq;
+      dg[static_cast<size_t>(i) * r + b] = u_i * (qq - w) + w * (scale * wbar[b] - wu);
+    }
+    return;
+  }
+  float a[CPMTP_MAX_R];
+  float acc[CPMTP_MAX_R];   // sum_s up_s q_s[b]
+  float up_sum = 0.f;
   for (int b = 0; b < r; ++b) {
+    a[b] = logw[static_cast<size_t>(i) * r + b];
+    acc[b] = 0.f;
+  }
+  // forward over s: weighted posteriors, parked in coef[i, s, :]
+  for (int s = 0; s < n; ++s) {
+    float m = -INFINITY;
+    for (int b = 0; b < r; ++b) {
+      const size_t row = static_cast<size_t>(i) * K + s * r + b;
+      a[b] += tgt[row] - lse[row];
+      m = fmaxf(m, a[b]);
+    }
+    float tot = 0.f;
+    for (int b = 0; b < r; ++b) tot += expf(a[b] - m);
+    const float inv = 1.0f / tot;
+    const float u_s = up[static_cast<size_t>(i) * n + s];
+    up_sum += u_s;
+    for (int b = 0; b < r; ++b) {
+      const float wq = u_s * expf(a[b] - m) * inv;
+      coef[static_cast<size_t>(i) * K + s * r + b] = wq;
+      acc[b] += wq;
+    }
+  }
+  // suffix sums over s, in place
+  for (int b = 0; b < r; ++b) {
+    float run = 0.f;
+    for (int s = n - 1; s >= 0; --s) {
+      run += coef[static_cast<size_t>(i) * K + s * r + b];
+      coef[static_cast<size_t>(i) * K + s * r + b] = run;
+    }
     const float w = expf(logw[static_cast<size_t>(i) * r + b]);
-    const float qq = q[static_cast<size_t>(i) * r + b];
-    coef[static_cast<size_t>(i) * r + b] = u_i * qq;
-    dg[static_cast<size_t>(i) * r + b] = u_i * (qq - w) + w * (scale * wbar[b] - wu);
+    dg[static_cast<size_t>(i) * r + b] = acc[b] - up_sum * w + w * (scale * wbar[b] - wu);
   }
 }
 

@@ -211,3 +211,35 @@ def test_backward_skips_outputs_that_are_not_asked_for(skip):
             assert torch.equal(part[key], full[key]), key
     with pytest.raises(binding.CpmtpError):
         binding.backward(*dev, saved, skip=("dh", "dW_head", "dE", "dW_g"))
+
+
+def test_backward_of_per_token_objective_matches_oracle():
+    """Weights on the prefix log-probabilities (CPMTP_FLAG_PER_TOKEN): a discounted per-token cross-entropy."""
+    from paper_2410_17765_b200 import binding
+
+    shape = synth.Shape(N=90, d=256, V=1300, n=4, r=5)
+    inp = synth.make_inputs(shape, seed=6, weight_scale=2.0)
+    gamma = 0.8
+    wts = torch.zeros((shape.N, shape.n), dtype=torch.float32)
+    for k in range(shape.n):
+        wts[:, k] -= gamma ** k / shape.N
+        if k > 0:
+            wts[:, k - 1] += gamma ** k / shape.N
+    ref = cp_head.backward(inp.h, inp.W_head, inp.E, inp.W_g, inp.x, shape.n, shape.r, aux_coef=0.5,
+                           dloss_dprefix=wts.numpy())
+    dev = to_dev(inp)
+    saved = binding.Saved.alloc(binding.make_shape(shape.N, shape.d, shape.V, shape.n, shape.r))
+    binding.forward(*dev, aux_coef=0.5, saved=saved)
+    g = binding.backward(*dev, saved, aux_coef=0.5, dloss_dprefix=wts.cuda())
+    torch.cuda.synchronize()
+    for key, want in (("dh", ref.dh), ("dW_head", ref.dW_head), ("dE", ref.dE), ("dW_g", ref.dW_g)):
+        assert rel_l2(g[key].float().cpu().numpy(), want) <= GRAD_TOL, (key, rel_l2(g[key].float().cpu().numpy(), want))
+    # full head, same objective
+    W_full = synth.make_full_head(shape, seed=6, weight_scale=3.0)
+    reff = cp_head.backward_full(inp.h, W_full, inp.W_g, inp.x, shape.n, shape.r, dloss_dprefix=wts.numpy())
+    saved_f = binding.Saved.alloc_full(binding.make_shape(shape.N, shape.d, shape.V, shape.n, shape.r))
+    binding.forward_full(dev[0], W_full.cuda(), dev[3], dev[4], saved=saved_f)
+    gf = binding.backward_full(dev[0], W_full.cuda(), dev[3], dev[4], saved_f, dloss_dprefix=wts.cuda())
+    torch.cuda.synchronize()
+    for key, want in (("dh", reff.dh), ("dW_full", reff.dW_full), ("dW_g", reff.dW_g)):
+        assert rel_l2(gf[key].float().cpu().numpy(), want) <= GRAD_TOL, key
