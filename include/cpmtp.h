@@ -76,6 +76,11 @@ enum {
  * sum_i sum_s dloss_dlogp[i, s] * log P(x[i, 0..s]).  The discounted per-token cross-entropy of the
  * fine-tuning loss (Eq. 14 and the sum after it, CE_k = log P(x[0..k-1]) - log P(x[0..k])) is of this form. */
 #define CPMTP_FLAG_PER_TOKEN 2u
+/* Do not keep the projected hidden states between the passes: cpmtp_forward leaves saved->z
+ * untouched (it may be NULL) and cpmtp_backward recomputes z in its workspace (which grows by
+ * N*n*r*d*2 bytes while the saved state shrinks by as much; +2*N*n*r*d*d flop).  Set the flag in
+ * both calls and in the workspace query. */
+#define CPMTP_FLAG_RECOMPUTE_Z 4u
 
 typedef struct cpmtp_shape {
   int32_t N;        /* positions */

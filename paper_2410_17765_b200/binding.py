@@ -18,6 +18,7 @@ from .build import LIB_PATH
 OP_FORWARD, OP_BACKWARD, OP_SCORE, OP_SAMPLE, OP_FORWARD_FULL, OP_BACKWARD_FULL = 0, 1, 2, 3, 4, 5
 FLAG_AUX = 1
 FLAG_PER_TOKEN = 2
+FLAG_RECOMPUTE_Z = 4
 
 EXPORTS = [
     "cpmtp_version", "cpmtp_status_string", "cpmtp_workspace_bytes", "cpmtp_forward", "cpmtp_backward",
@@ -168,7 +169,7 @@ class Saved:
 
     def c_struct(self) -> CSaved:
         return CSaved(self.lse.data_ptr(), self.tgt.data_ptr(), self.logw.data_ptr(), self.q.data_ptr(),
-                      self.wbar.data_ptr(), self.z.data_ptr())
+                      self.wbar.data_ptr(), self.z.data_ptr() if self.z is not None else None)
 
 
 def _shape_of(h, W_head, E, W_g, x, aux_coef) -> CShape:
@@ -185,10 +186,14 @@ def _shape_of(h, W_head, E, W_g, x, aux_coef) -> CShape:
 
 def forward(h, W_head, E, W_g, x, *, aux_coef: Optional[float] = None, saved: Optional[Saved] = None,
             want_loss: bool = True, want_counts: bool = False, workspace: Optional[torch.Tensor] = None,
-            dev_status: Optional[torch.Tensor] = None, out: Optional[dict] = None) -> dict:
-    """cpmtp_forward on device tensors; returns {"logp", "loss", "counts"} (device tensors)."""
+            dev_status: Optional[torch.Tensor] = None, out: Optional[dict] = None,
+            recompute_z: bool = False) -> dict:
+    """cpmtp_forward on device tensors; returns {"logp", "loss", "counts"} (device tensors).
+    recompute_z: do not keep z in `saved` (CPMTP_FLAG_RECOMPUTE_Z; pass the same to backward)."""
     lib = load_library()
     shape = _shape_of(h, W_head, E, W_g, x, aux_coef)
+    if recompute_z:
+        shape.flags |= FLAG_RECOMPUTE_Z
     dev = h.device
     if workspace is None:
         workspace = alloc_workspace(workspace_bytes(shape, OP_FORWARD), dev)
@@ -212,12 +217,15 @@ def forward(h, W_head, E, W_g, x, *, aux_coef: Optional[float] = None, saved: Op
 def backward(h, W_head, E, W_g, x, saved: Saved, *, aux_coef: Optional[float] = None,
              dloss_dlogp: Optional[torch.Tensor] = None, workspace: Optional[torch.Tensor] = None,
              dev_status: Optional[torch.Tensor] = None, out: Optional[dict] = None,
-             skip: tuple = (), dloss_dprefix: Optional[torch.Tensor] = None) -> dict:
+             skip: tuple = (), dloss_dprefix: Optional[torch.Tensor] = None,
+             recompute_z: bool = False) -> dict:
     """cpmtp_backward on device tensors; returns {"dh", "dW_head", "dE", "dW_g"} (bf16 device tensors).
     Names listed in `skip` are not computed (passed as NULL).  dloss_dprefix [N, n] fp32 selects the
     per-token objective sum_i sum_s dloss_dprefix[i, s] * log P(x[i, 0..s]) (CPMTP_FLAG_PER_TOKEN)."""
     lib = load_library()
     shape = _shape_of(h, W_head, E, W_g, x, aux_coef)
+    if recompute_z:
+        shape.flags |= FLAG_RECOMPUTE_Z
     if dloss_dprefix is not None:
         assert dloss_dlogp is None and dloss_dprefix.shape == (shape.N, shape.n) and dloss_dprefix.dtype == torch.float32
         shape.flags |= FLAG_PER_TOKEN

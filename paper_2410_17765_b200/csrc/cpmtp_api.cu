@@ -149,7 +149,7 @@ FwdLayout fwd_layout(const cpmtp_shape& s, int sms) {
 }
 
 struct BwdLayout {
-  size_t coef, dg, dz, G, dE32, dwg_part, total;
+  size_t coef, dg, dz, zre, G, dE32, dwg_part, total;
   int K, M, ldg, chunk_rows, chunks, dwg_slices, dwg_rows_per_slice;
 };
 
@@ -175,6 +175,7 @@ BwdLayout bwd_layout(const cpmtp_shape& s) {
   L.coef = take(sizeof(float) * static_cast<size_t>(s.N) * L.K);
   L.dg = take(sizeof(float) * s.N * s.r);
   L.dz = take(2ull * L.M * s.d);
+  L.zre = take((s.flags & CPMTP_FLAG_RECOMPUTE_Z) ? 2ull * L.M * s.d : 0);   // z recomputed instead of saved
   L.G = take(2ull * L.chunk_rows * L.ldg);
   L.dE32 = take(L.chunks > 1 ? sizeof(float) * static_cast<size_t>(s.V) * s.d : 0);
   L.dwg_part = take(sizeof(float) * static_cast<size_t>(L.dwg_slices) * s.r * s.d);
@@ -351,7 +352,8 @@ int run_forward(const cpmtp_shape& s, const uint16_t* h, const uint16_t* W_head,
   float* wbar = saved ? saved->wbar : reinterpret_cast<float*>(ws + L.wbar);
   float* lse = saved ? saved->lse : reinterpret_cast<float*>(ws + L.lse);
   float* tgt = saved ? saved->tgt : reinterpret_cast<float*>(ws + L.tgt);
-  uint16_t* z = saved ? static_cast<uint16_t*>(saved->z) : reinterpret_cast<uint16_t*>(ws + L.z);
+  const bool keep_z = saved != nullptr && !(s.flags & CPMTP_FLAG_RECOMPUTE_Z);
+  uint16_t* z = keep_z ? static_cast<uint16_t*>(saved->z) : reinterpret_cast<uint16_t*>(ws + L.z);
   float* tgt_part = reinterpret_cast<float*>(ws + L.tgt_part);
   float* part_m = reinterpret_cast<float*>(ws + L.part_m);
   float* part_l = reinterpret_cast<float*>(ws + L.part_l);
@@ -426,8 +428,8 @@ int check_common(const cpmtp_shape* shape, const void* h, const void* W_head, co
   return CPMTP_OK;
 }
 
-int check_saved(const cpmtp_saved* sv) {
-  if (!sv->lse || !sv->tgt || !sv->logw || !sv->q || !sv->wbar || !sv->z) return CPMTP_ERR_NULL;
+int check_saved(const cpmtp_saved* sv, bool need_z = true) {
+  if (!sv->lse || !sv->tgt || !sv->logw || !sv->q || !sv->wbar || (need_z && !sv->z)) return CPMTP_ERR_NULL;
   if (!aligned(sv->z, 16) || !aligned(sv->lse, 4) || !aligned(sv->tgt, 4) || !aligned(sv->logw, 4) ||
       !aligned(sv->q, 4) || !aligned(sv->wbar, 4))
     return CPMTP_ERR_ALIGN;
@@ -540,7 +542,7 @@ int cpmtp_forward(const cpmtp_shape* shape, const void* h, const void* W_head, c
   if (rc != CPMTP_OK) return rc;
   if (logp == nullptr) return CPMTP_ERR_NULL;
   if (saved != nullptr) {
-    const int rs = check_saved(saved);
+    const int rs = check_saved(saved, !(shape->flags & CPMTP_FLAG_RECOMPUTE_Z));
     if (rs != CPMTP_OK) return rs;
   }
   const FwdLayout L = fwd_layout(*shape, di->sms);
@@ -824,7 +826,8 @@ int cpmtp_backward(const cpmtp_shape* shape, const void* h, const void* W_head, 
   if (rc != CPMTP_OK) return rc;
   if (saved == nullptr) return CPMTP_ERR_NULL;
   if (!dh && !dW_head && !dE && !dW_g) return CPMTP_ERR_NULL;   // nothing asked for
-  const int rs = check_saved(saved);
+  const bool recompute_z = (shape->flags & CPMTP_FLAG_RECOMPUTE_Z) != 0;
+  const int rs = check_saved(saved, !recompute_z);
   if (rs != CPMTP_OK) return rs;
   if (!aligned(dh, 16) || !aligned(dW_head, 16) || !aligned(dE, 16) || !aligned(dW_g, 16)) return CPMTP_ERR_ALIGN;
   const bool need_dz = dh != nullptr || dW_head != nullptr;   // dz feeds only these two
@@ -839,7 +842,8 @@ int cpmtp_backward(const cpmtp_shape* shape, const void* h, const void* W_head, 
   uint16_t* G = reinterpret_cast<uint16_t*>(ws + L.G);
   float* dE32 = reinterpret_cast<float*>(ws + L.dE32);
   float* dwg_part = reinterpret_cast<float*>(ws + L.dwg_part);
-  const uint16_t* z = static_cast<const uint16_t*>(saved->z);
+  const uint16_t* z = recompute_z ? reinterpret_cast<const uint16_t*>(ws + L.zre)
+                                  : static_cast<const uint16_t*>(saved->z);
   const uint16_t* Eb = static_cast<const uint16_t*>(E);
   const int sms = di->sms;
   const int K = L.K, d = s.d, V = s.V;
@@ -848,6 +852,11 @@ int cpmtp_backward(const cpmtp_shape* shape, const void* h, const void* W_head, 
   const int per_token = (s.flags & CPMTP_FLAG_PER_TOKEN) ? 1 : 0;
   if (per_token && dloss_dlogp == nullptr) return CPMTP_ERR_NULL;
 
+  if (recompute_z) {   // z[N, K*d] = h W_cat^T again: the same MMAs and the same rounding as in the forward pass
+    ProfScope prof(CPMTP_STAGE_PROJ, st);
+    EpiStoreBf16<kBN, false>::Params ep{reinterpret_cast<uint16_t*>(ws + L.zre), nullptr, nullptr, s.N, ncols, ncols, 0};
+    CPMTP_TRY((gemm_auto<false, false, EpiStoreBf16<kBN, false>>(h, d, W_head, d, s.N, ncols, d, 8192, ep, dev_status, sms, st)));
+  }
   {
     ProfScope prof(CPMTP_STAGE_COEFF, st);
     coeff_kernel<<<(s.N + 127) / 128, 128, 0, st>>>(saved->q, saved->logw, saved->wbar, saved->lse, saved->tgt,

@@ -243,3 +243,25 @@ def test_backward_of_per_token_objective_matches_oracle():
     torch.cuda.synchronize()
     for key, want in (("dh", reff.dh), ("dW_full", reff.dW_full), ("dW_g", reff.dW_g)):
         assert rel_l2(gf[key].float().cpu().numpy(), want) <= GRAD_TOL, key
+
+
+def test_recomputing_z_in_the_backward_gives_identical_gradients():
+    from paper_2410_17765_b200 import binding
+
+    shape = CASES["wide"]["shape"]
+    inp = synth.make_inputs(shape, seed=0)
+    dev = to_dev(inp)
+    cs = binding.make_shape(shape.N, shape.d, shape.V, shape.n, shape.r)
+    saved = binding.Saved.alloc(cs)
+    f1 = binding.forward(*dev, saved=saved)
+    g1 = binding.backward(*dev, saved)
+    lean = binding.Saved.alloc(cs)
+    lean.z = None                                  # nothing of size N*K*d is kept between the passes
+    f2 = binding.forward(*dev, saved=lean, recompute_z=True)
+    g2 = binding.backward(*dev, lean, recompute_z=True)
+    torch.cuda.synchronize()
+    assert torch.equal(f1["logp"], f2["logp"])
+    for key in ("dh", "dW_head", "dE", "dW_g"):
+        assert torch.equal(g1[key], g2[key]), key
+    with pytest.raises(binding.CpmtpError):
+        binding.backward(*dev, lean)               # z missing and no flag
