@@ -325,6 +325,10 @@ cudaError_t gemm_auto(const void* A, uint64_t a_ld, const void* B, uint64_t b_ld
                       cudaStream_t stream) {
   const int n_tiles = (n_cols + kBN - 1) / kBN;
   const int k_blocks = static_cast<int>((kdim + kBK - 1) / kBK);
+  if (const char* env = std::getenv("CPMTP_GEMM_GROUP_ROWS")) {   // tuning knob
+    const int v = std::atoi(env);
+    if (v >= kWideBM) group_rows = v;
+  }
   if (use_wide(m_rows, kdim)) {
     const int m_tiles = static_cast<int>((m_rows + kWideBM - 1) / kWideBM);
     const Sched sc = make_sched(m_tiles, n_tiles, n_tiles, group_rows / kWideBM, k_blocks);
