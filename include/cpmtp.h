@@ -35,7 +35,8 @@
  *    CPMTP_BWD_CHUNK_ROWS / CPMTP_BWD_CHUNK_HEADS (rows / heads of logit gradients
  *    recomputed at a time in the backward passes; also changes the workspace the
  *    backward needs, so set it before querying cpmtp_workspace_bytes),
- *    CPMTP_LSE_GROUP_MB and CPMTP_LSE_SPLITS (schedule of the fused unembedding),
+ *    CPMTP_LSE_GROUP_MB, CPMTP_LSE_SPLITS and CPMTP_LSE_GROUP_TILES (schedule of the
+ *    fused unembedding),
  *    CPMTP_GEMM_GROUP_ROWS (rows swept together by the other GEMMs).
  */
 #ifndef CPMTP_H

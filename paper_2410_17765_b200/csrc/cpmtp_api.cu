@@ -113,7 +113,24 @@ Sched sched_lse(int m_tiles, int n_tiles, int M, int V, int d, int bm, int slots
     const int v = std::atoi(env);
     if (v >= 1 && v <= s_max) best_s = v;
   }
-  const int group = static_cast<long long>(m_tiles) * best_s >= sms ? (sms / best_s) : m_tiles;
+  int group = static_cast<long long>(m_tiles) * best_s >= sms ? (sms / best_s) : m_tiles;
+  if (bm > kBM && m_tiles >= 8) {
+    // 256-row tiles (d >= 4096): measured on B200, short units in the raster of the plain GEMMs beat
+    // the long lock-stepped sweeps above: 8 row tiles (2048 rows) x 125 vocabulary ranges ran the
+    // unembedding 20 % faster at V = 128256 and 4-9 % faster at V = 32000 (A/B within one process).
+    // Range counts that make a group a whole number of waves (e.g. 148) were clearly worse.
+    group = 8;
+    best_s = n_tiles < 125 ? n_tiles : 125;
+    if ((static_cast<long long>(group) * best_s) % sms == 0 && best_s > 1) --best_s;
+    if (const char* env2 = std::getenv("CPMTP_LSE_SPLITS")) {
+      const int v = std::atoi(env2);
+      if (v >= 1 && v <= n_tiles) best_s = v;
+    }
+  }
+  if (const char* env = std::getenv("CPMTP_LSE_GROUP_TILES")) {   // tuning knob: force the row group
+    const int v = std::atoi(env);
+    if (v >= 1) group = v;
+  }
   return make_sched(m_tiles, n_tiles, best_s, group < 1 ? 1 : group, d / kBK);
 }
 
