@@ -37,7 +37,8 @@
  *    backward needs, so set it before querying cpmtp_workspace_bytes),
  *    CPMTP_LSE_GROUP_MB, CPMTP_LSE_SPLITS and CPMTP_LSE_GROUP_TILES (schedule of the
  *    fused unembedding),
- *    CPMTP_GEMM_GROUP_ROWS (rows swept together by the other GEMMs).
+ *    CPMTP_GEMM_GROUP_ROWS (rows swept together by the other GEMMs), CPMTP_WIDE_MIN_K
+ *    (shortest contraction that gets 256-row tiles).
  */
 #ifndef CPMTP_H
 #define CPMTP_H

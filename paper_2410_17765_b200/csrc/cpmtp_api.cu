@@ -68,7 +68,14 @@ inline bool aligned(const void* p, size_t a) { return (reinterpret_cast<uintptr_
 // Wide (256-row) tiles move a third fewer operand bytes per flop but cannot overlap their
 // epilogue with the next tile's MMAs, so they pay when the contraction is long enough to
 // amortise it; otherwise 128-row tiles with the double-buffered accumulator are used.
-bool use_wide(long long rows, long long kdim) { return rows >= 2 * kWideBM && kdim >= 4096; }
+bool use_wide(long long rows, long long kdim) {
+  long long min_k = 4096;
+  if (const char* env = std::getenv("CPMTP_WIDE_MIN_K")) {   // tuning knob
+    const long long v = std::atoll(env);
+    if (v >= 64) min_k = v;
+  }
+  return rows >= 2 * kWideBM && kdim >= min_k;
+}
 
 // Column-split schedule of the fused unembedding: `group` row tiles x `splits`
 // vocabulary ranges run concurrently, so the rows' z tiles stay L2-resident while
