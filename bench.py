@@ -102,11 +102,18 @@ class ClockSampler:
                 "samples": len(sm), "reasons": sorted(reasons)}
 
 
-def flops_per_position(s, kind):
+def flops_per_position(s, kind, skip=()):
     K = s.n * s.r
     fwd = 2 * K * (s.d * s.d + s.V * s.d) + 2 * s.r * s.d
     if kind == "full_fwd_bwd":
         return 3 * (2 * K * s.V * s.d + 2 * s.r * s.d)
+    if kind == "fwd_bwd" and skip:
+        # forward + dz always; dE, dW_head, dh only when asked for
+        total = fwd + 2 * K * s.V * s.d
+        total += 0 if "dE" in skip else 2 * K * s.V * s.d
+        total += 0 if "dW_head" in skip else 2 * K * s.d * s.d
+        total += 0 if "dh" in skip else 2 * K * s.d * s.d
+        return total
     return fwd if kind != "fwd_bwd" else 3 * fwd
 
 
@@ -312,7 +319,7 @@ def run_ours(args, rank: int, world: int, local_rank: int):
     roof["peak_source"] = peaks["src"]
     roof["avg_launch_ms"] = avg_ms
     roof["algorithmic_per_launch"] = alg
-    total_flops = flops_per_position(shape, kind) * positions * args.steps
+    total_flops = flops_per_position(shape, kind, skip) * positions * args.steps
     n_sub = oracle_sample_size(shape, kind)
     sec_per_pos, n_sub = oracle_seconds_per_position(inp, kind, aux, n_sub)
     line = {
