@@ -25,3 +25,12 @@ def pytest_collection_modifyitems(config, items):
     for item in items:
         if "gpu" in item.keywords:
             item.add_marker(skip)
+
+
+@pytest.fixture(scope="session", autouse=True)
+def _built_library():
+    """Compile libcpmtp.so once per session if it is missing or older than its sources."""
+    from paper_2410_17765_b200 import build
+
+    build.build()
+    yield
