@@ -140,3 +140,18 @@ def subsample_positions(inp: Inputs, idx: torch.Tensor) -> Inputs:
     sub = Shape(N=int(idx.numel()), d=s.d, V=s.V, n=s.n, r=s.r)
     return Inputs(shape=sub, h=inp.h[idx].contiguous(), W_head=inp.W_head, E=inp.E,
                   W_g=inp.W_g, x=inp.x[idx].contiguous())
+
+
+def make_teacher_logits(shape: Shape, x: torch.Tensor, seed: int = 0, *, std: float = 2.0,
+                        target_bump: float = 4.0) -> torch.Tensor:
+    """Teacher logits [N, n, V] bf16 for the distillation objective: N(0, std) noise with the
+    sequence's own token raised by ``target_bump`` (a frozen base model mostly agrees with its
+    training data).  Drawn in slabs of positions from a generator of its own."""
+    gen = torch.Generator(device="cpu")
+    gen.manual_seed(seed + 104729)
+    s = shape
+    T = _randn_bf16(gen, (s.N, s.n, s.V), std)
+    if target_bump != 0.0:
+        idx = x.to(torch.int64).unsqueeze(-1)
+        T.scatter_(2, idx, (T.gather(2, idx).float() + target_bump).to(torch.bfloat16))
+    return T
