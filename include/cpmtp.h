@@ -70,7 +70,9 @@ enum {
   CPMTP_OP_SCORE = 2,
   CPMTP_OP_SAMPLE = 3,
   CPMTP_OP_FORWARD_FULL = 4,
-  CPMTP_OP_BACKWARD_FULL = 5
+  CPMTP_OP_BACKWARD_FULL = 5,
+  CPMTP_OP_DISTILL_FORWARD = 6,
+  CPMTP_OP_DISTILL_BACKWARD = 7
 };
 
 /* flags */
@@ -215,6 +217,56 @@ int cpmtp_backward_full(const cpmtp_shape* shape, const void* h, const void* W_f
                         size_t workspace_bytes, int32_t* dev_status, cpmtp_stream stream);
 
 /*
+ * Fine-tuning objective with distillation (fine-tuning section, Eq. 14 and the sum after it).
+ * For every position i and predicted token k the head's distribution of that token given the
+ * tokens before it (taken from the sequence),
+ *   p^d[i,k,:] = sum_a pi[i,k,a] P^(k)(. | a),   pi[i,k,a] ~ w_a prod_{t<k} P^(t)(x[i,t] | a)
+ * (the conditional of the sampling section), is compared with a frozen model's p^c[i,k,:] =
+ * softmax(teacher[i,k,:]):
+ *   kl[i,k] = sum_v p^d(v) log(p^d(v) / p^c(v))                 (head first, as printed)
+ *   ce[i,k] = -log p^d[i,k,x[i,k]] = logp_prefix[i,k-1] - logp_prefix[i,k]
+ *   loss    = (1/N) sum_i sum_k gamma^k (beta kl[i,k] + (1 - beta) ce[i,k])   (k = 0..n-1)
+ *             (+ aux_coef * sum_a wbar_a^2 with CPMTP_FLAG_AUX).
+ * The printed conditioning of p^d is garbled and the printed sum runs over "0..d"; the reading
+ * above is the one the surrounding text supports.  The paper sets beta = 0.9.
+ *   teacher [N,n,V] bf16 logits (a constant added to a row changes nothing), 16-byte aligned.
+ *   logp [N], logp_prefix [N,n], dsaved->kl [N,n] fp32 out; loss [1] fp32 out or NULL.
+ *   saved and dsaved are required and are filled for cpmtp_distill_backward.
+ * The vocabulary is swept twice: the fused log-sum-exp pass of cpmtp_forward, then a pass in which
+ * the r experts of a (position, token) pair occupy adjacent accumulator rows (padded to a power of
+ * two) and are mixed across lanes, so p^d and the logits are never written to memory either.
+ * Workspace: CPMTP_OP_DISTILL_FORWARD.  CPMTP_FLAG_RECOMPUTE_Z is honoured as in cpmtp_forward.
+ */
+typedef struct cpmtp_distill_saved {
+  float* lse_t;  /* [N, n]    logsumexp_v teacher                                  */
+  float* logpi;  /* [N, n*r]  log pi                                               */
+  float* pm;     /* [N, n*r]  sum_v pi P^(k)(v | a) log(p^d(v) / p^c(v))           */
+  float* kl;     /* [N, n]    the KL terms (sum_a pm)                              */
+} cpmtp_distill_saved;
+
+int cpmtp_distill_forward(const cpmtp_shape* shape, const void* h, const void* W_head, const void* E,
+                          const void* W_g, const int32_t* x, const void* teacher, float beta, float gamma,
+                          float* logp, float* logp_prefix, float* loss, const cpmtp_saved* saved,
+                          const cpmtp_distill_saved* dsaved, void* workspace, size_t workspace_bytes,
+                          int32_t* dev_status, cpmtp_stream stream);
+
+/*
+ * Gradient of  sum_i sum_k ( dloss_dprefix[i,k] * logp_prefix[i,k] + dloss_dkl[i,k] * kl[i,k] )
+ * (+ the balance term with CPMTP_FLAG_AUX) with respect to h, W_head, E and W_g.  Either weight
+ * array may be NULL and then takes the values that make the sum equal the loss of
+ * cpmtp_distill_forward for (beta, gamma): dloss_dkl = beta gamma^k / N and
+ * dloss_dprefix = (1 - beta)(gamma^(k+1) [k+1 < n] - gamma^k) / N.
+ * The KL term reaches the logits directly and, through the expert weights pi, the target terms of
+ * the earlier tokens and the gate.  Outputs and the NULL-able gradient pointers as for
+ * cpmtp_backward.  Workspace: CPMTP_OP_DISTILL_BACKWARD.
+ */
+int cpmtp_distill_backward(const cpmtp_shape* shape, const void* h, const void* W_head, const void* E,
+                           const void* W_g, const int32_t* x, const void* teacher, const cpmtp_saved* saved,
+                           const cpmtp_distill_saved* dsaved, float beta, float gamma, const float* dloss_dprefix,
+                           const float* dloss_dkl, void* dh, void* dW_head, void* dE, void* dW_g, void* workspace,
+                           size_t workspace_bytes, int32_t* dev_status, cpmtp_stream stream);
+
+/*
  * Verify drafts (draft-then-verify of the Preliminaries; speculative-decoding section).
  * accepted [N] int32 out: how many leading tokens of each draft are kept.
  *  - Greedy (base_tokens != NULL): the longest common prefix of draft [N,n] and the
@@ -300,6 +352,8 @@ enum {
   CPMTP_STAGE_DH,
   CPMTP_STAGE_DW_G,
   CPMTP_STAGE_DRAFT_STEP,    /* per-token selection passes of cpmtp_sample_draft */
+  CPMTP_STAGE_TEACHER_LSE,   /* logsumexp_V of the teacher logits + expert weights per token (Eq. 14) */
+  CPMTP_STAGE_KL,            /* second unembedding pass: KL term of Eq. 14 */
   CPMTP_STAGE_COUNT
 };
 int cpmtp_profile_begin(void);

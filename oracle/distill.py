@@ -33,10 +33,11 @@ import numpy as np
 from . import cp_head as cp
 
 
-def conditional_log_probs(h, W_head, E, W_g, x, n: int, r: int):
+def conditional_log_probs(h, W_head, E, W_g, x, n: int, r: int, *, round_z: bool = False):
     """log p^d[i, k, v] and log pi[i, k, a] (mixture weights before token k), teacher-forced on x.
 
-    Also returns log P^(k)(v | a) as logP[i, k, a, v] for the gradient."""
+    Also returns log P^(k)(v | a) as logP[i, k, a, v] for the gradient.  round_z rounds the projected
+    hidden states to bf16 first (explanatory mode only, as in cp_head.factor_log_probs)."""
     hd, Ed, xi = cp._f64(h), cp._f64(E), cp._i64(x)
     N = hd.shape[0]
     V = Ed.shape[0]
@@ -44,7 +45,10 @@ def conditional_log_probs(h, W_head, E, W_g, x, n: int, r: int):
     logP = np.empty((N, n, r, V))
     for k in range(n * r):
         s, a = divmod(k, r)
-        S = cp.head_projection(hd, W_head[k]) @ Ed.T
+        z = cp.head_projection(hd, W_head[k])
+        if round_z:
+            z = cp.round_to_bf16(z)
+        S = z @ Ed.T
         logP[:, s, a, :] = S - cp.logsumexp(S, axis=1)[:, None]
     rows = np.arange(N)
     lb = logw.copy()
@@ -66,9 +70,9 @@ class Distill:
 
 
 def forward(h, W_head, E, W_g, x, teacher, n: int, r: int, *, beta: float = 0.9, gamma: float = 1.0,
-            aux_coef: float = 0.0) -> Distill:
+            aux_coef: float = 0.0, round_z: bool = False) -> Distill:
     """Eq. 14 and the discounted sum after it."""
-    logpd, _, _ = conditional_log_probs(h, W_head, E, W_g, x, n, r)
+    logpd, _, _ = conditional_log_probs(h, W_head, E, W_g, x, n, r, round_z=round_z)
     T = cp._f64(teacher)
     logpc = T - cp.logsumexp(T, axis=2)[:, :, None]
     pd = np.exp(logpd)

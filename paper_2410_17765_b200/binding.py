@@ -16,6 +16,7 @@ import torch
 from .build import LIB_PATH
 
 OP_FORWARD, OP_BACKWARD, OP_SCORE, OP_SAMPLE, OP_FORWARD_FULL, OP_BACKWARD_FULL = 0, 1, 2, 3, 4, 5
+OP_DISTILL_FORWARD, OP_DISTILL_BACKWARD = 6, 7
 FLAG_AUX = 1
 FLAG_PER_TOKEN = 2
 FLAG_RECOMPUTE_Z = 4
@@ -25,12 +26,13 @@ EXPORTS = [
     "cpmtp_score_draft", "cpmtp_host_staging_bytes", "cpmtp_forward_host", "cpmtp_profile_begin",
     "cpmtp_profile_end", "cpmtp_score_draft_static", "cpmtp_sample_draft",
     "cpmtp_forward_full", "cpmtp_backward_full", "cpmtp_verify_draft",
+    "cpmtp_distill_forward", "cpmtp_distill_backward",
 ]
 
 STATIC_SCRATCH_BYTES = 4 << 20
 
 STAGES = ["gate", "proj", "lse", "mixture", "finalize", "coeff", "logit_grad", "dz", "de", "de_convert",
-          "dw_head", "dh", "dw_g", "draft_step"]
+          "dw_head", "dh", "dw_g", "draft_step", "teacher_lse", "kl"]
 
 
 class CShape(ctypes.Structure):
@@ -41,6 +43,11 @@ class CShape(ctypes.Structure):
 class CSaved(ctypes.Structure):
     _fields_ = [("lse", ctypes.c_void_p), ("tgt", ctypes.c_void_p), ("logw", ctypes.c_void_p),
                 ("q", ctypes.c_void_p), ("wbar", ctypes.c_void_p), ("z", ctypes.c_void_p)]
+
+
+class CDistillSaved(ctypes.Structure):
+    _fields_ = [("lse_t", ctypes.c_void_p), ("logpi", ctypes.c_void_p), ("pm", ctypes.c_void_p),
+                ("kl", ctypes.c_void_p)]
 
 
 _lib = None
@@ -83,6 +90,13 @@ def load_library() -> ctypes.CDLL:
     lib.cpmtp_verify_draft.argtypes = [ctypes.c_int32, ctypes.c_int32, i32p, i32p, fp, fp, fp, i32p, vp]
     lib.cpmtp_score_draft_static.restype = ctypes.c_int
     lib.cpmtp_score_draft_static.argtypes = [shp, vp, vp, vp, vp, i32p, fp, fp, i32p, vp]
+    dsp = ctypes.POINTER(CDistillSaved)
+    lib.cpmtp_distill_forward.restype = ctypes.c_int
+    lib.cpmtp_distill_forward.argtypes = [shp, vp, vp, vp, vp, i32p, vp, ctypes.c_float, ctypes.c_float, fp, fp, fp,
+                                          svp, dsp, vp, sz, i32p, vp]
+    lib.cpmtp_distill_backward.restype = ctypes.c_int
+    lib.cpmtp_distill_backward.argtypes = [shp, vp, vp, vp, vp, i32p, vp, svp, dsp, ctypes.c_float, ctypes.c_float,
+                                           fp, fp, vp, vp, vp, vp, vp, sz, i32p, vp]
     lib.cpmtp_profile_begin.restype = ctypes.c_int
     lib.cpmtp_profile_end.restype = ctypes.c_int
     lib.cpmtp_profile_end.argtypes = [ctypes.POINTER(ctypes.c_float), ctypes.POINTER(ctypes.c_int32), ctypes.c_int]
@@ -410,3 +424,85 @@ def forward_host(h_host, W_head, E, W_g, x_host, logp_host, loss_host, *, aux_co
                                 _ptr(workspace), workspace.numel(),
                                 _ptr(dev_status), _stream())
     _check(rc)
+
+
+@dataclass
+class DistillSaved:
+    """Results of cpmtp_distill_forward kept for cpmtp_distill_backward (device tensors); `kl` is also
+    the entry point's output, KL(p^d_k, p^c_k) per (position, token)."""
+    lse_t: torch.Tensor
+    logpi: torch.Tensor
+    pm: torch.Tensor
+    kl: torch.Tensor
+
+    @staticmethod
+    def alloc(shape: CShape, device="cuda") -> "DistillSaved":
+        f = dict(dtype=torch.float32, device=device)
+        K = shape.n * shape.r
+        return DistillSaved(lse_t=torch.empty((shape.N, shape.n), **f), logpi=torch.empty((shape.N, K), **f),
+                            pm=torch.empty((shape.N, K), **f), kl=torch.empty((shape.N, shape.n), **f))
+
+    def c_struct(self) -> CDistillSaved:
+        return CDistillSaved(self.lse_t.data_ptr(), self.logpi.data_ptr(), self.pm.data_ptr(), self.kl.data_ptr())
+
+
+def _check_teacher(teacher, shape: CShape) -> None:
+    assert teacher.shape == (shape.N, shape.n, shape.V) and teacher.dtype == torch.bfloat16 and teacher.is_contiguous()
+
+
+def distill_forward(h, W_head, E, W_g, x, teacher, saved: Saved, dsaved: DistillSaved, *, beta: float = 0.9,
+                    gamma: float = 1.0, aux_coef: Optional[float] = None, want_loss: bool = True,
+                    workspace: Optional[torch.Tensor] = None, dev_status: Optional[torch.Tensor] = None,
+                    out: Optional[dict] = None, recompute_z: bool = False) -> dict:
+    """cpmtp_distill_forward; returns {"logp", "logp_prefix", "kl", "loss"} (device tensors; kl is dsaved.kl)."""
+    lib = load_library()
+    shape = _shape_of(h, W_head, E, W_g, x, aux_coef)
+    _check_teacher(teacher, shape)
+    if recompute_z:
+        shape.flags |= FLAG_RECOMPUTE_Z
+    dev = h.device
+    if workspace is None:
+        workspace = alloc_workspace(workspace_bytes(shape, OP_DISTILL_FORWARD), dev)
+    res = out if out is not None else {}
+    res.setdefault("logp", torch.empty(shape.N, dtype=torch.float32, device=dev))
+    res.setdefault("logp_prefix", torch.empty((shape.N, shape.n), dtype=torch.float32, device=dev))
+    if want_loss:
+        res.setdefault("loss", torch.empty(1, dtype=torch.float32, device=dev))
+    res["kl"] = dsaved.kl
+    cs, ds = saved.c_struct(), dsaved.c_struct()
+    rc = lib.cpmtp_distill_forward(ctypes.byref(shape), _ptr(h), _ptr(W_head), _ptr(E), _ptr(W_g), _ptr(x),
+                                   _ptr(teacher), ctypes.c_float(beta), ctypes.c_float(gamma), _ptr(res["logp"]),
+                                   _ptr(res["logp_prefix"]), _ptr(res.get("loss")) if want_loss else None,
+                                   ctypes.byref(cs), ctypes.byref(ds), _ptr(workspace), workspace.numel(),
+                                   _ptr(dev_status), _stream())
+    _check(rc)
+    return res
+
+
+def distill_backward(h, W_head, E, W_g, x, teacher, saved: Saved, dsaved: DistillSaved, *, beta: float = 0.9,
+                     gamma: float = 1.0, aux_coef: Optional[float] = None,
+                     dloss_dprefix: Optional[torch.Tensor] = None, dloss_dkl: Optional[torch.Tensor] = None,
+                     workspace: Optional[torch.Tensor] = None, dev_status: Optional[torch.Tensor] = None,
+                     out: Optional[dict] = None, skip: tuple = (), recompute_z: bool = False) -> dict:
+    """cpmtp_distill_backward; returns {"dh", "dW_head", "dE", "dW_g"} (bf16 device tensors)."""
+    lib = load_library()
+    shape = _shape_of(h, W_head, E, W_g, x, aux_coef)
+    _check_teacher(teacher, shape)
+    if recompute_z:
+        shape.flags |= FLAG_RECOMPUTE_Z
+    for w in (dloss_dprefix, dloss_dkl):
+        assert w is None or (w.shape == (shape.N, shape.n) and w.dtype == torch.float32 and w.is_contiguous())
+    if workspace is None:
+        workspace = alloc_workspace(workspace_bytes(shape, OP_DISTILL_BACKWARD), h.device)
+    res = out if out is not None else {}
+    for name, ref in (("dh", h), ("dW_head", W_head), ("dE", E), ("dW_g", W_g)):
+        if name not in res and name not in skip:
+            res[name] = torch.empty_like(ref)
+    cs, ds = saved.c_struct(), dsaved.c_struct()
+    rc = lib.cpmtp_distill_backward(ctypes.byref(shape), _ptr(h), _ptr(W_head), _ptr(E), _ptr(W_g), _ptr(x),
+                                    _ptr(teacher), ctypes.byref(cs), ctypes.byref(ds), ctypes.c_float(beta),
+                                    ctypes.c_float(gamma), _ptr(dloss_dprefix), _ptr(dloss_dkl), _ptr(res.get("dh")),
+                                    _ptr(res.get("dW_head")), _ptr(res.get("dE")), _ptr(res.get("dW_g")),
+                                    _ptr(workspace), workspace.numel(), _ptr(dev_status), _stream())
+    _check(rc)
+    return res

@@ -10,7 +10,8 @@ PKG_DIR = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(PKG_DIR, "csrc")
 LIB_PATH = os.path.join(PKG_DIR, "libcpmtp.so")
 SOURCES = ["cpmtp_api.cu"]
-HEADERS = ["ptx.cuh", "tmap.cuh", "tc_gemm.cuh", "epilogues.cuh", "small_kernels.cuh", "sampler_kernels.cuh"]
+HEADERS = ["ptx.cuh", "tmap.cuh", "tc_gemm.cuh", "epilogues.cuh", "small_kernels.cuh", "sampler_kernels.cuh",
+           "distill_epilogues.cuh", "distill_kernels.cuh"]
 
 
 def _nvcc() -> str:

@@ -8,6 +8,8 @@
 #include <cstdlib>
 #include <vector>
 
+#include "distill_epilogues.cuh"
+#include "distill_kernels.cuh"
 #include "epilogues.cuh"
 #include "sampler_kernels.cuh"
 #include "small_kernels.cuh"
@@ -173,22 +175,31 @@ FwdLayout fwd_layout(const cpmtp_shape& s, int sms) {
 }
 
 struct BwdLayout {
-  size_t coef, dg, dz, zre, G, dE32, dwg_part, total;
+  size_t coef, dg, dz, zre, G, dE32, dwg_part, uk, total;
   int K, M, ldg, chunk_rows, chunks, dwg_slices, dwg_rows_per_slice;
 };
 
-BwdLayout bwd_layout(const cpmtp_shape& s) {
+// Group size of the distillation passes: r padded to a power of two (lanes of a warp).
+inline int padded_rank(int r) {
+  int R = 1;
+  while (R < r) R <<= 1;
+  return R;
+}
+
+// `quantum`: chunks of recomputed logit gradients hold a multiple of this many rows (whole row
+// tiles: 128 rows, or 128 / R groups of r rows for the grouped distillation pass).
+BwdLayout bwd_layout(const cpmtp_shape& s, int quantum = kBM, bool distill = false) {
   BwdLayout L;
   L.K = s.n * s.r;
   L.M = s.N * L.K;
   L.ldg = (s.V + 63) / 64 * 64;
-  long long rows = static_cast<long long>(kLogitGradBudgetBytes / (2ull * L.ldg)) / kBM * kBM;
+  long long rows = static_cast<long long>(kLogitGradBudgetBytes / (2ull * L.ldg)) / quantum * quantum;
   if (const char* env = std::getenv("CPMTP_BWD_CHUNK_ROWS")) {
     const long long v = std::atoll(env);
-    if (v >= kBM) rows = v / kBM * kBM;
+    if (v >= quantum) rows = v / quantum * quantum;
   }
-  if (rows < kBM) rows = kBM;
-  const long long m_pad = (static_cast<long long>(L.M) + kBM - 1) / kBM * kBM;
+  if (rows < quantum) rows = quantum;
+  const long long m_pad = (static_cast<long long>(L.M) + quantum - 1) / quantum * quantum;
   if (rows > m_pad) rows = m_pad;
   L.chunk_rows = static_cast<int>(rows);
   L.chunks = static_cast<int>((L.M + rows - 1) / rows);
@@ -203,6 +214,32 @@ BwdLayout bwd_layout(const cpmtp_shape& s) {
   L.G = take(2ull * L.chunk_rows * L.ldg);
   L.dE32 = take(L.chunks > 1 ? sizeof(float) * static_cast<size_t>(s.V) * s.d : 0);
   L.dwg_part = take(sizeof(float) * static_cast<size_t>(L.dwg_slices) * s.r * s.d);
+  L.uk = take(distill ? sizeof(float) * static_cast<size_t>(s.N) * s.n : 0);
+  L.total = off;
+  return L;
+}
+
+// Distillation forward: the plain forward pass, then the grouped KL pass over the vocabulary.
+struct DistillLayout {
+  FwdLayout fwd;
+  size_t part, total;
+  Sched sched;
+  int R, gpt, groups;   // padded rank, groups per 128-row tile, N * n
+};
+
+DistillLayout distill_layout(const cpmtp_shape& s, int sms) {
+  DistillLayout L;
+  L.fwd = fwd_layout(s, sms);
+  L.R = padded_rank(s.r);
+  L.gpt = kBM / L.R;
+  L.groups = s.N * s.n;
+  const int m_tiles = (L.groups + L.gpt - 1) / L.gpt;
+  const int n_tiles = (s.V + kBN - 1) / kBN;
+  L.sched = sched_lse(m_tiles, n_tiles, m_tiles * kBM, s.V, s.d, kBM, sms);
+  L.sched.a_groups = L.gpt;
+  size_t off = align_up(L.fwd.total);
+  auto take = [&](size_t bytes) { size_t o = off; off = align_up(off + bytes); return o; };
+  L.part = take(sizeof(float) * static_cast<size_t>(L.fwd.M) * L.sched.n_splits);
   L.total = off;
   return L;
 }
@@ -323,10 +360,18 @@ SampleLayout sample_layout(const cpmtp_shape& s, int sms) {
 template <class Cfg, class Epi>
 cudaError_t launch_gemm(const void* A, uint64_t a_rows, uint64_t a_ld, const void* B, uint64_t b_rows,
                         uint64_t b_ld, uint64_t kdim, const Sched& sched, const typename Epi::Params& ep,
-                        int* dev_status, int sms, cudaStream_t stream) {
+                        int* dev_status, int sms, cudaStream_t stream, int a_group_rows = 0) {
   static bool attr_set[64] = {};
   CUtensorMap tA, tB;
-  if (!make_operand_tmap(&tA, A, Cfg::A_MN, a_rows, kdim, a_ld, Cfg::A_ROWS * Cfg::MB)) return cudaErrorInvalidValue;
+  if (sched.a_groups > 0) {
+    // grouped rows: a_rows = groups * a_group_rows, every group padded to 128 / a_groups tile rows
+    if (Cfg::A_MN || Cfg::MB != 1 || Cfg::A_ROWS != kBM || a_group_rows < 1) return cudaErrorInvalidValue;
+    if (!make_grouped_tmap_bf16(&tA, A, kdim, a_group_rows, a_rows / a_group_rows, a_ld, kBM / sched.a_groups,
+                                sched.a_groups))
+      return cudaErrorInvalidValue;
+  } else if (!make_operand_tmap(&tA, A, Cfg::A_MN, a_rows, kdim, a_ld, Cfg::A_ROWS * Cfg::MB)) {
+    return cudaErrorInvalidValue;
+  }
   if (!make_operand_tmap(&tB, B, Cfg::B_MN, b_rows, kdim, b_ld, Cfg::BN)) return cudaErrorInvalidValue;
   constexpr int smem = gemm_smem_bytes<Cfg, Epi>();
   int dev = 0;
@@ -492,6 +537,196 @@ static int sms_or_default() {
   return (di != nullptr && di->sms > 0) ? di->sms : 148;
 }
 
+
+// The two grouped passes, instantiated for every padded rank R (a power of two, 1..32).
+template <int RR>
+static cudaError_t distill_kl_r(const uint16_t* z, long long rows, int d, const uint16_t* E, int V, const Sched& sc,
+                                float* part, const float* lse, const float* logpi, const float* lse_t,
+                                const uint16_t* T, int groups, int r, int* dev_status, int sms, cudaStream_t st) {
+  typename EpiKl<kBN, RR>::Params ep{part, lse, logpi, lse_t, T, groups, r, V, sc.n_splits, V % 8 == 0 ? 1 : 0};
+  return launch_gemm<CfgKK, EpiKl<kBN, RR>>(z, rows, d, E, V, d, d, sc, ep, dev_status, sms, st, r);
+}
+
+static cudaError_t launch_distill_kl(int R, const uint16_t* z, long long rows, int d, const uint16_t* E, int V,
+                                     const Sched& sc, float* part, const float* lse, const float* logpi,
+                                     const float* lse_t, const uint16_t* T, int groups, int r, int* dev_status,
+                                     int sms, cudaStream_t st) {
+  switch (R) {
+    case 1: return distill_kl_r<1>(z, rows, d, E, V, sc, part, lse, logpi, lse_t, T, groups, r, dev_status, sms, st);
+    case 2: return distill_kl_r<2>(z, rows, d, E, V, sc, part, lse, logpi, lse_t, T, groups, r, dev_status, sms, st);
+    case 4: return distill_kl_r<4>(z, rows, d, E, V, sc, part, lse, logpi, lse_t, T, groups, r, dev_status, sms, st);
+    case 8: return distill_kl_r<8>(z, rows, d, E, V, sc, part, lse, logpi, lse_t, T, groups, r, dev_status, sms, st);
+    case 16: return distill_kl_r<16>(z, rows, d, E, V, sc, part, lse, logpi, lse_t, T, groups, r, dev_status, sms, st);
+    case 32: return distill_kl_r<32>(z, rows, d, E, V, sc, part, lse, logpi, lse_t, T, groups, r, dev_status, sms, st);
+    default: return cudaErrorInvalidValue;
+  }
+}
+
+template <int RR>
+static cudaError_t distill_grad_r(const uint16_t* z, long long rows, int d, const uint16_t* E, const Sched& sc,
+                                  const typename EpiDistillGrad<kBN, RR>::Params& ep, int r, int* dev_status, int sms,
+                                  cudaStream_t st) {
+  // the column tiles that cover V also cover the padding columns [V, ldg), which are written as zero
+  return launch_gemm<CfgKK, EpiDistillGrad<kBN, RR>>(z, rows, d, E, ep.V, d, d, sc, ep, dev_status, sms, st, r);
+}
+
+static cudaError_t launch_distill_grad(int R, const uint16_t* z, long long rows, int d, const uint16_t* E, int V,
+                                       const Sched& sc, uint16_t* G, const cpmtp_saved* saved, const float* coef,
+                                       const cpmtp_distill_saved* ds, const float* uk, const uint16_t* T,
+                                       const int32_t* x, long long grp0, int groups, int r, int ldg,
+                                       int* dev_status, int sms, cudaStream_t st) {
+  // identical parameter blocks for every R
+  const EpiDistillGrad<kBN, 1>::Params p1{G, saved->lse, coef, ds->logpi, ds->pm, uk, ds->lse_t, T, x,
+                                          grp0, groups, r, V, ldg, V % 8 == 0 ? 1 : 0};
+  auto as = [&](auto tag) {
+    typename decltype(tag)::Params q{p1.G, p1.lse, p1.coef, p1.logpi, p1.pm, p1.uk, p1.lse_t, p1.T, p1.x,
+                                     p1.grp0, p1.groups, p1.r, p1.V, p1.ldg, p1.vec};
+    return q;
+  };
+  switch (R) {
+    case 1: return distill_grad_r<1>(z, rows, d, E, sc, as(EpiDistillGrad<kBN, 1>{}), r, dev_status, sms, st);
+    case 2: return distill_grad_r<2>(z, rows, d, E, sc, as(EpiDistillGrad<kBN, 2>{}), r, dev_status, sms, st);
+    case 4: return distill_grad_r<4>(z, rows, d, E, sc, as(EpiDistillGrad<kBN, 4>{}), r, dev_status, sms, st);
+    case 8: return distill_grad_r<8>(z, rows, d, E, sc, as(EpiDistillGrad<kBN, 8>{}), r, dev_status, sms, st);
+    case 16: return distill_grad_r<16>(z, rows, d, E, sc, as(EpiDistillGrad<kBN, 16>{}), r, dev_status, sms, st);
+    case 32: return distill_grad_r<32>(z, rows, d, E, sc, as(EpiDistillGrad<kBN, 32>{}), r, dev_status, sms, st);
+    default: return cudaErrorInvalidValue;
+  }
+}
+
+// What the distillation objective adds to the backward pass (nullptr: plain log-likelihood).
+struct DistillCtx {
+  const uint16_t* teacher;          // [N, n, V] bf16
+  const cpmtp_distill_saved* ds;
+  const float* dloss_dkl;           // [N, n] or nullptr (weights of Eq. 14 from beta, gamma)
+  float beta, gamma;
+};
+
+// Backward pipeline shared by cpmtp_backward and cpmtp_distill_backward.
+static int backward_impl(const cpmtp_shape* shape, const void* h, const void* W_head, const void* E, const void* W_g,
+                         const int32_t* x, const cpmtp_saved* saved, const float* dloss_dlogp, void* dh,
+                         void* dW_head, void* dE, void* dW_g, void* workspace, size_t workspace_bytes,
+                         int32_t* dev_status, cpmtp_stream stream, const DistillCtx* dc) {
+  DeviceInfo* di = nullptr;
+  const int rc = check_common(shape, h, W_head, E, W_g, x, workspace, &di);
+  if (rc != CPMTP_OK) return rc;
+  if (saved == nullptr) return CPMTP_ERR_NULL;
+  if (!dh && !dW_head && !dE && !dW_g) return CPMTP_ERR_NULL;   // nothing asked for
+  const bool recompute_z = (shape->flags & CPMTP_FLAG_RECOMPUTE_Z) != 0;
+  const int rs = check_saved(saved, !recompute_z);
+  if (rs != CPMTP_OK) return rs;
+  if (!aligned(dh, 16) || !aligned(dW_head, 16) || !aligned(dE, 16) || !aligned(dW_g, 16)) return CPMTP_ERR_ALIGN;
+  const bool need_dz = dh != nullptr || dW_head != nullptr;   // dz feeds only these two
+  const cpmtp_shape& s = *shape;
+  const int R = padded_rank(s.r);
+  const int gpt = kBM / R;   // groups per row tile of the grouped pass
+  const BwdLayout L = dc != nullptr ? bwd_layout(s, gpt * s.r, true) : bwd_layout(s);
+  if (workspace_bytes < L.total) return CPMTP_ERR_WORKSPACE;
+  cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
+  uint8_t* ws = static_cast<uint8_t*>(workspace);
+  float* coef = reinterpret_cast<float*>(ws + L.coef);
+  float* dg = reinterpret_cast<float*>(ws + L.dg);
+  uint16_t* dz = reinterpret_cast<uint16_t*>(ws + L.dz);
+  uint16_t* G = reinterpret_cast<uint16_t*>(ws + L.G);
+  float* dE32 = reinterpret_cast<float*>(ws + L.dE32);
+  float* dwg_part = reinterpret_cast<float*>(ws + L.dwg_part);
+  const uint16_t* z = recompute_z ? reinterpret_cast<const uint16_t*>(ws + L.zre)
+                                  : static_cast<const uint16_t*>(saved->z);
+  const uint16_t* Eb = static_cast<const uint16_t*>(E);
+  const int sms = di->sms;
+  const int K = L.K, d = s.d, V = s.V;
+  const int ncols = K * d;
+  const float aux = (s.flags & CPMTP_FLAG_AUX) ? s.aux_coef : 0.f;
+  const int per_token = (s.flags & CPMTP_FLAG_PER_TOKEN) ? 1 : 0;
+  if (per_token && dloss_dlogp == nullptr && dc == nullptr) return CPMTP_ERR_NULL;
+  float* uk = reinterpret_cast<float*>(ws + L.uk);
+
+  if (recompute_z) {   // z[N, K*d] = h W_cat^T again: the same MMAs and the same rounding as in the forward pass
+    ProfScope prof(CPMTP_STAGE_PROJ, st);
+    EpiStoreBf16<kBN, false>::Params ep{reinterpret_cast<uint16_t*>(ws + L.zre), nullptr, nullptr, s.N, ncols, ncols, 0};
+    CPMTP_TRY((gemm_auto<false, false, EpiStoreBf16<kBN, false>>(h, d, W_head, d, s.N, ncols, d, 8192, ep, dev_status, sms, st)));
+  }
+  {
+    ProfScope prof(CPMTP_STAGE_COEFF, st);
+    if (dc != nullptr) {
+      distill_coeff_kernel<<<(s.N + 127) / 128, 128, 0, st>>>(saved->logw, saved->wbar, saved->lse, saved->tgt,
+                                                             dc->ds->logpi, dc->ds->pm, dc->ds->kl, dloss_dlogp,
+                                                             dc->dloss_dkl, dc->beta, dc->gamma, coef, dg, uk, s.N,
+                                                             s.n, s.r, aux);
+    } else {
+      coeff_kernel<<<(s.N + 127) / 128, 128, 0, st>>>(saved->q, saved->logw, saved->wbar, saved->lse, saved->tgt,
+                                                     dloss_dlogp, per_token, coef, dg, s.N, s.n, s.r, aux);
+    }
+    CPMTP_TRY(cudaGetLastError());
+  }
+
+  for (int c = 0; c < L.chunks; ++c) {
+    const long long row0 = static_cast<long long>(c) * L.chunk_rows;
+    const int rows = static_cast<int>((L.M - row0) < L.chunk_rows ? (L.M - row0) : L.chunk_rows);
+    const uint16_t* zc = z + row0 * d;
+    // recompute logits tile by tile -> G = dloss/dS (bf16), never more than one chunk
+    if (dc != nullptr) {
+      ProfScope prof(CPMTP_STAGE_LOGIT_GRAD, st);
+      const int groups = rows / s.r;   // chunks hold whole groups
+      Sched sc = make_sched((groups + gpt - 1) / gpt, (V + kBN - 1) / kBN, (V + kBN - 1) / kBN, 2048 / kBM, d / kBK);
+      sc.a_groups = gpt;
+      CPMTP_TRY(launch_distill_grad(R, zc, rows, d, Eb, V, sc, G, saved, coef, dc->ds, uk, dc->teacher, x,
+                                    row0 / s.r, groups, s.r, L.ldg, dev_status, sms, st));
+    } else if (need_dz || dE != nullptr) {
+      ProfScope prof(CPMTP_STAGE_LOGIT_GRAD, st);
+      EpiLogitGrad<kBN>::Params ep{G, saved->lse, coef, x, row0, rows, L.ldg, V, K, s.n, s.r};
+      CPMTP_TRY((gemm_auto<false, false, EpiLogitGrad<kBN>>(zc, d, Eb, d, rows, V, d, 2048, ep, dev_status, sms, st)));
+    }
+    // dz[rows, d] = G[rows, V] * E[V, d]
+    if (need_dz) {
+      ProfScope prof(CPMTP_STAGE_DZ, st);
+      EpiStoreBf16<kBN, false>::Params ep{dz + row0 * d, nullptr, nullptr, rows, d, d, 0};
+      CPMTP_TRY((gemm_auto<false, true, EpiStoreBf16<kBN, false>>(G, L.ldg, Eb, d, rows, d, V, 2048, ep, dev_status, sms, st)));
+    }
+    // dE[V, d] (+)= G^T[V, rows] * z[rows, d]
+    if (dE != nullptr) {
+      ProfScope prof(CPMTP_STAGE_DE, st);
+      if (L.chunks == 1) {
+        EpiStoreBf16<kBN, false>::Params ep{static_cast<uint16_t*>(dE), nullptr, nullptr, V, d, d, 0};
+        CPMTP_TRY((gemm_auto<true, true, EpiStoreBf16<kBN, false>>(G, L.ldg, zc, d, V, d, rows, 2048, ep, dev_status, sms, st)));
+      } else {
+        EpiAccumF32<kBN>::Params ep{dE32, V, d, d, c > 0 ? 1 : 0};
+        CPMTP_TRY((gemm_auto<true, true, EpiAccumF32<kBN>>(G, L.ldg, zc, d, V, d, rows, 2048, ep, dev_status, sms, st)));
+      }
+    }
+  }
+  if (L.chunks > 1 && dE != nullptr) {
+    ProfScope prof(CPMTP_STAGE_DE_CONVERT, st);
+    f32_to_bf16_kernel<<<sms * 8, 256, 0, st>>>(dE32, static_cast<uint16_t*>(dE), static_cast<size_t>(V) * d);
+    CPMTP_TRY(cudaGetLastError());
+  }
+  // dW_head[K*d, d] = dz^T[K*d, N] * h[N, d]
+  if (dW_head != nullptr) {
+    ProfScope prof(CPMTP_STAGE_DW_HEAD, st);
+    EpiStoreBf16<kBN, false>::Params ep{static_cast<uint16_t*>(dW_head), nullptr, nullptr, ncols, d, d, 0};
+    CPMTP_TRY((gemm_auto<true, true, EpiStoreBf16<kBN, false>>(dz, ncols, h, d, ncols, d, s.N, 2048, ep, dev_status, sms, st)));
+  }
+  // dh[N, d] = dz[N, K*d] * W_cat[K*d, d] + dg * W_g
+  if (dh != nullptr) {
+    ProfScope prof(CPMTP_STAGE_DH, st);
+    EpiStoreBf16<kBN, true>::Params ep{static_cast<uint16_t*>(dh), dg, static_cast<const uint16_t*>(W_g), s.N, d, d, s.r};
+    CPMTP_TRY((gemm_auto<false, true, EpiStoreBf16<kBN, true>>(dz, ncols, W_head, d, s.N, d, ncols, 2048, ep, dev_status, sms, st)));
+  }
+  // dW_g[r, d] = dg^T * h
+  if (dW_g != nullptr) {
+    ProfScope prof(CPMTP_STAGE_DW_G, st);
+    dim3 grid((d + 127) / 128, L.dwg_slices);
+    dwg_partial_kernel<CPMTP_MAX_R><<<grid, 128, 0, st>>>(dg, static_cast<const uint16_t*>(h), dwg_part, s.N, d, s.r,
+                                                          L.dwg_rows_per_slice);
+    CPMTP_TRY(cudaGetLastError());
+    dwg_reduce_kernel<<<(s.r * d + 255) / 256, 256, 0, st>>>(dwg_part, static_cast<uint16_t*>(dW_g), L.dwg_slices,
+                                                            s.r, d);
+    CPMTP_TRY(cudaGetLastError());
+  }
+  return CPMTP_OK;
+}
+
+
 extern "C" {
 
 int cpmtp_version(void) { return 100; }
@@ -552,6 +787,9 @@ size_t cpmtp_workspace_bytes(const cpmtp_shape* shape, int op) {
     case CPMTP_OP_SAMPLE: return sample_layout(*shape, sms).total;
     case CPMTP_OP_FORWARD_FULL: return full_layout(*shape, sms).total;
     case CPMTP_OP_BACKWARD_FULL: return full_bwd_layout(*shape).total;
+    case CPMTP_OP_DISTILL_FORWARD: return distill_layout(*shape, sms).total;
+    case CPMTP_OP_DISTILL_BACKWARD:
+      return bwd_layout(*shape, kBM / padded_rank(shape->r) * shape->r, true).total;
     default: return 0;
   }
 }
@@ -845,110 +1083,81 @@ int cpmtp_forward_host(const cpmtp_shape* shape, const void* h_host, const void*
   return CPMTP_OK;
 }
 
+int cpmtp_distill_forward(const cpmtp_shape* shape, const void* h, const void* W_head, const void* E,
+                          const void* W_g, const int32_t* x, const void* teacher, float beta, float gamma,
+                          float* logp, float* logp_prefix, float* loss, const cpmtp_saved* saved,
+                          const cpmtp_distill_saved* dsaved, void* workspace, size_t workspace_bytes,
+                          int32_t* dev_status, cpmtp_stream stream) {
+  DeviceInfo* di = nullptr;
+  const int rc = check_common(shape, h, W_head, E, W_g, x, workspace, &di);
+  if (rc != CPMTP_OK) return rc;
+  if (!teacher || !logp || !logp_prefix || !saved || !dsaved) return CPMTP_ERR_NULL;
+  if (!dsaved->lse_t || !dsaved->logpi || !dsaved->pm || !dsaved->kl) return CPMTP_ERR_NULL;
+  if (!aligned(teacher, 16)) return CPMTP_ERR_ALIGN;
+  const cpmtp_shape& s = *shape;
+  const bool recompute_z = (s.flags & CPMTP_FLAG_RECOMPUTE_Z) != 0;
+  const int rs = check_saved(saved, !recompute_z);
+  if (rs != CPMTP_OK) return rs;
+  const DistillLayout L = distill_layout(s, di->sms);
+  if (workspace_bytes < L.total) return CPMTP_ERR_WORKSPACE;
+  cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
+  uint8_t* ws = static_cast<uint8_t*>(workspace);
+  const uint16_t* Tb = static_cast<const uint16_t*>(teacher);
+  // Eq. 9 with the prefix scores (the cross-entropy part of Eq. 14), lse / tgt / logw / wbar / z kept
+  const int rf = run_forward(s, static_cast<const uint16_t*>(h), static_cast<const uint16_t*>(W_head),
+                             static_cast<const uint16_t*>(E), static_cast<const uint16_t*>(W_g), x, logp, nullptr, saved,
+                             nullptr, logp_prefix, ws, L.fwd, dev_status, di->sms, st);
+  if (rf != CPMTP_OK) return rf;
+  const uint16_t* z = recompute_z ? reinterpret_cast<const uint16_t*>(ws + L.fwd.z)
+                                  : static_cast<const uint16_t*>(saved->z);
+  {
+    ProfScope prof(CPMTP_STAGE_TEACHER_LSE, st);
+    teacher_lse_kernel<<<L.groups, kTeacherThreads, 0, st>>>(Tb, s.V, dsaved->lse_t);
+    CPMTP_TRY(cudaGetLastError());
+    distill_pi_kernel<<<(s.N + 127) / 128, 128, 0, st>>>(saved->logw, saved->lse, saved->tgt, dsaved->logpi, s.N, s.n,
+                                                        s.r);
+    CPMTP_TRY(cudaGetLastError());
+  }
+  float* part = reinterpret_cast<float*>(ws + L.part);
+  {
+    ProfScope prof(CPMTP_STAGE_KL, st);
+    CPMTP_TRY(launch_distill_kl(L.R, z, L.fwd.M, s.d, static_cast<const uint16_t*>(E), s.V, L.sched, part, saved->lse,
+                                dsaved->logpi, dsaved->lse_t, Tb, L.groups, s.r, dev_status, di->sms, st));
+  }
+  {
+    ProfScope prof(CPMTP_STAGE_FINALIZE, st);
+    distill_merge_kernel<<<(L.groups + 3) / 4, 128, 0, st>>>(part, L.sched.n_splits, dsaved->pm, dsaved->kl, L.groups,
+                                                            s.r);
+    CPMTP_TRY(cudaGetLastError());
+    if (loss != nullptr) {
+      const float aux = (s.flags & CPMTP_FLAG_AUX) ? s.aux_coef : 0.f;
+      distill_loss_kernel<<<1, kDistillLossThreads, 0, st>>>(logp_prefix, dsaved->kl, saved->wbar, nullptr, nullptr,
+                                                            beta, gamma, aux, s.N, s.n, s.r, loss);
+      CPMTP_TRY(cudaGetLastError());
+    }
+  }
+  return CPMTP_OK;
+}
+
+int cpmtp_distill_backward(const cpmtp_shape* shape, const void* h, const void* W_head, const void* E,
+                           const void* W_g, const int32_t* x, const void* teacher, const cpmtp_saved* saved,
+                           const cpmtp_distill_saved* dsaved, float beta, float gamma, const float* dloss_dprefix,
+                           const float* dloss_dkl, void* dh, void* dW_head, void* dE, void* dW_g, void* workspace,
+                           size_t workspace_bytes, int32_t* dev_status, cpmtp_stream stream) {
+  if (!teacher || !dsaved) return CPMTP_ERR_NULL;
+  if (!dsaved->lse_t || !dsaved->logpi || !dsaved->pm || !dsaved->kl) return CPMTP_ERR_NULL;
+  if (!aligned(teacher, 16)) return CPMTP_ERR_ALIGN;
+  DistillCtx dc{static_cast<const uint16_t*>(teacher), dsaved, dloss_dkl, beta, gamma};
+  return backward_impl(shape, h, W_head, E, W_g, x, saved, dloss_dprefix, dh, dW_head, dE, dW_g, workspace,
+                       workspace_bytes, dev_status, stream, &dc);
+}
+
 int cpmtp_backward(const cpmtp_shape* shape, const void* h, const void* W_head, const void* E, const void* W_g,
                    const int32_t* x, const cpmtp_saved* saved, const float* dloss_dlogp, void* dh, void* dW_head,
                    void* dE, void* dW_g, void* workspace, size_t workspace_bytes, int32_t* dev_status,
                    cpmtp_stream stream) {
-  DeviceInfo* di = nullptr;
-  const int rc = check_common(shape, h, W_head, E, W_g, x, workspace, &di);
-  if (rc != CPMTP_OK) return rc;
-  if (saved == nullptr) return CPMTP_ERR_NULL;
-  if (!dh && !dW_head && !dE && !dW_g) return CPMTP_ERR_NULL;   // nothing asked for
-  const bool recompute_z = (shape->flags & CPMTP_FLAG_RECOMPUTE_Z) != 0;
-  const int rs = check_saved(saved, !recompute_z);
-  if (rs != CPMTP_OK) return rs;
-  if (!aligned(dh, 16) || !aligned(dW_head, 16) || !aligned(dE, 16) || !aligned(dW_g, 16)) return CPMTP_ERR_ALIGN;
-  const bool need_dz = dh != nullptr || dW_head != nullptr;   // dz feeds only these two
-  const cpmtp_shape& s = *shape;
-  const BwdLayout L = bwd_layout(s);
-  if (workspace_bytes < L.total) return CPMTP_ERR_WORKSPACE;
-  cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
-  uint8_t* ws = static_cast<uint8_t*>(workspace);
-  float* coef = reinterpret_cast<float*>(ws + L.coef);
-  float* dg = reinterpret_cast<float*>(ws + L.dg);
-  uint16_t* dz = reinterpret_cast<uint16_t*>(ws + L.dz);
-  uint16_t* G = reinterpret_cast<uint16_t*>(ws + L.G);
-  float* dE32 = reinterpret_cast<float*>(ws + L.dE32);
-  float* dwg_part = reinterpret_cast<float*>(ws + L.dwg_part);
-  const uint16_t* z = recompute_z ? reinterpret_cast<const uint16_t*>(ws + L.zre)
-                                  : static_cast<const uint16_t*>(saved->z);
-  const uint16_t* Eb = static_cast<const uint16_t*>(E);
-  const int sms = di->sms;
-  const int K = L.K, d = s.d, V = s.V;
-  const int ncols = K * d;
-  const float aux = (s.flags & CPMTP_FLAG_AUX) ? s.aux_coef : 0.f;
-  const int per_token = (s.flags & CPMTP_FLAG_PER_TOKEN) ? 1 : 0;
-  if (per_token && dloss_dlogp == nullptr) return CPMTP_ERR_NULL;
-
-  if (recompute_z) {   // z[N, K*d] = h W_cat^T again: the same MMAs and the same rounding as in the forward pass
-    ProfScope prof(CPMTP_STAGE_PROJ, st);
-    EpiStoreBf16<kBN, false>::Params ep{reinterpret_cast<uint16_t*>(ws + L.zre), nullptr, nullptr, s.N, ncols, ncols, 0};
-    CPMTP_TRY((gemm_auto<false, false, EpiStoreBf16<kBN, false>>(h, d, W_head, d, s.N, ncols, d, 8192, ep, dev_status, sms, st)));
-  }
-  {
-    ProfScope prof(CPMTP_STAGE_COEFF, st);
-    coeff_kernel<<<(s.N + 127) / 128, 128, 0, st>>>(saved->q, saved->logw, saved->wbar, saved->lse, saved->tgt,
-                                                   dloss_dlogp, per_token, coef, dg, s.N, s.n, s.r, aux);
-    CPMTP_TRY(cudaGetLastError());
-  }
-
-  for (int c = 0; c < L.chunks; ++c) {
-    const long long row0 = static_cast<long long>(c) * L.chunk_rows;
-    const int rows = static_cast<int>((L.M - row0) < L.chunk_rows ? (L.M - row0) : L.chunk_rows);
-    const uint16_t* zc = z + row0 * d;
-    // recompute logits tile by tile -> G = dloss/dS (bf16), never more than one chunk
-    if (need_dz || dE != nullptr) {
-      ProfScope prof(CPMTP_STAGE_LOGIT_GRAD, st);
-      EpiLogitGrad<kBN>::Params ep{G, saved->lse, coef, x, row0, rows, L.ldg, V, K, s.n, s.r};
-      CPMTP_TRY((gemm_auto<false, false, EpiLogitGrad<kBN>>(zc, d, Eb, d, rows, V, d, 2048, ep, dev_status, sms, st)));
-    }
-    // dz[rows, d] = G[rows, V] * E[V, d]
-    if (need_dz) {
-      ProfScope prof(CPMTP_STAGE_DZ, st);
-      EpiStoreBf16<kBN, false>::Params ep{dz + row0 * d, nullptr, nullptr, rows, d, d, 0};
-      CPMTP_TRY((gemm_auto<false, true, EpiStoreBf16<kBN, false>>(G, L.ldg, Eb, d, rows, d, V, 2048, ep, dev_status, sms, st)));
-    }
-    // dE[V, d] (+)= G^T[V, rows] * z[rows, d]
-    if (dE != nullptr) {
-      ProfScope prof(CPMTP_STAGE_DE, st);
-      if (L.chunks == 1) {
-        EpiStoreBf16<kBN, false>::Params ep{static_cast<uint16_t*>(dE), nullptr, nullptr, V, d, d, 0};
-        CPMTP_TRY((gemm_auto<true, true, EpiStoreBf16<kBN, false>>(G, L.ldg, zc, d, V, d, rows, 2048, ep, dev_status, sms, st)));
-      } else {
-        EpiAccumF32<kBN>::Params ep{dE32, V, d, d, c > 0 ? 1 : 0};
-        CPMTP_TRY((gemm_auto<true, true, EpiAccumF32<kBN>>(G, L.ldg, zc, d, V, d, rows, 2048, ep, dev_status, sms, st)));
-      }
-    }
-  }
-  if (L.chunks > 1 && dE != nullptr) {
-    ProfScope prof(CPMTP_STAGE_DE_CONVERT, st);
-    f32_to_bf16_kernel<<<sms * 8, 256, 0, st>>>(dE32, static_cast<uint16_t*>(dE), static_cast<size_t>(V) * d);
-    CPMTP_TRY(cudaGetLastError());
-  }
-  // dW_head[K*d, d] = dz^T[K*d, N] * h[N, d]
-  if (dW_head != nullptr) {
-    ProfScope prof(CPMTP_STAGE_DW_HEAD, st);
-    EpiStoreBf16<kBN, false>::Params ep{static_cast<uint16_t*>(dW_head), nullptr, nullptr, ncols, d, d, 0};
-    CPMTP_TRY((gemm_auto<true, true, EpiStoreBf16<kBN, false>>(dz, ncols, h, d, ncols, d, s.N, 2048, ep, dev_status, sms, st)));
-  }
-  // dh[N, d] = dz[N, K*d] * W_cat[K*d, d] + dg * W_g
-  if (dh != nullptr) {
-    ProfScope prof(CPMTP_STAGE_DH, st);
-    EpiStoreBf16<kBN, true>::Params ep{static_cast<uint16_t*>(dh), dg, static_cast<const uint16_t*>(W_g), s.N, d, d, s.r};
-    CPMTP_TRY((gemm_auto<false, true, EpiStoreBf16<kBN, true>>(dz, ncols, W_head, d, s.N, d, ncols, 2048, ep, dev_status, sms, st)));
-  }
-  // dW_g[r, d] = dg^T * h
-  if (dW_g != nullptr) {
-    ProfScope prof(CPMTP_STAGE_DW_G, st);
-    dim3 grid((d + 127) / 128, L.dwg_slices);
-    dwg_partial_kernel<CPMTP_MAX_R><<<grid, 128, 0, st>>>(dg, static_cast<const uint16_t*>(h), dwg_part, s.N, d, s.r,
-                                                          L.dwg_rows_per_slice);
-    CPMTP_TRY(cudaGetLastError());
-    dwg_reduce_kernel<<<(s.r * d + 255) / 256, 256, 0, st>>>(dwg_part, static_cast<uint16_t*>(dW_g), L.dwg_slices,
-                                                            s.r, d);
-    CPMTP_TRY(cudaGetLastError());
-  }
-  return CPMTP_OK;
+  return backward_impl(shape, h, W_head, E, W_g, x, saved, dloss_dlogp, dh, dW_head, dE, dW_g, workspace,
+                       workspace_bytes, dev_status, stream, nullptr);
 }
 
 }  // extern "C"

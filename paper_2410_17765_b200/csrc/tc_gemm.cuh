@@ -54,6 +54,9 @@ struct Sched {
   // (nt / seg_tiles) * seg_stride + (nt % seg_tiles) * BN instead of nt * BN.
   int seg_tiles;
   int seg_stride;
+  // Grouped rows of A (0 = off; K-major A, MB = 1 only): the A tensor map is 3-D [groups][r][K] and a
+  // row tile holds a_groups whole groups, each padded to 128 / a_groups rows (see make_grouped_tmap_bf16).
+  int a_groups;
 };
 
 inline Sched make_sched(int m_tiles, int n_tiles, int n_splits, int m_group, int k_blocks) {
@@ -70,6 +73,7 @@ inline Sched make_sched(int m_tiles, int n_tiles, int n_splits, int m_group, int
   s.units = ((m_tiles + m_group - 1) / m_group) * m_group * n_splits;
   s.seg_tiles = 0;
   s.seg_stride = 0;
+  s.a_groups = 0;
   return s;
 }
 
@@ -196,7 +200,11 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             const uint32_t b_dst = a_dst + Cfg::A_BYTES;
             if constexpr (!Cfg::A_MN) {
               // one box of A_ROWS * MB rows: block b lands at a_dst + b * A_BLOCK_BYTES
-              ptx::tma_load_2d(a_dst, &tmA, full_bar(s), kb * kBK, m_tile * Cfg::TILE_M);
+              if (sched.a_groups > 0) {
+                ptx::tma_load_3d(a_dst, &tmA, full_bar(s), kb * kBK, 0, m_tile * sched.a_groups);
+              } else {
+                ptx::tma_load_2d(a_dst, &tmA, full_bar(s), kb * kBK, m_tile * Cfg::TILE_M);
+              }
             } else {
 #pragma unroll
               for (int j = 0; j < Cfg::TILE_M / 64; ++j)

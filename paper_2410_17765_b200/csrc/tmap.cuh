@@ -1,4 +1,4 @@
-// Host-side construction of 2-D bf16 TMA tensor maps (128-byte swizzle).
+// Host-side construction of bf16 TMA tensor maps (128-byte swizzle).
 // The driver entry point is fetched at run time so the library has no link-time
 // dependency on libcuda.
 #pragma once
@@ -41,6 +41,24 @@ inline bool make_tmap_bf16(CUtensorMap* out, const void* base, uint64_t inner, u
                   CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                   CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
   return r == CUDA_SUCCESS;
+}
+
+// K-major A operand whose rows come in groups of `r` that are padded to `R` >= r tile rows:
+// matrix [groups * r, k] viewed as [groups][r][k]; a box holds 64 (k) x R x groups_per_box and the
+// rows r..R-1 of every group, like everything else out of range, read as zero.  The box lands in
+// shared memory as groups_per_box * R dense 128-byte rows, i.e. as an ordinary row tile.
+inline bool make_grouped_tmap_bf16(CUtensorMap* out, const void* base, uint64_t k, uint64_t r, uint64_t groups,
+                                   uint64_t ld, uint32_t R, uint32_t groups_per_box) {
+  EncodeTiledFn fn = get_encode_fn();
+  if (fn == nullptr) return false;
+  cuuint64_t dims[3] = {k, r, groups};
+  cuuint64_t strides[2] = {ld * 2, ld * 2 * r};
+  cuuint32_t box[3] = {64, R, groups_per_box};
+  cuuint32_t elem[3] = {1, 1, 1};
+  CUresult rc = fn(out, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(base), dims, strides, box, elem,
+                   CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                   CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return rc == CUDA_SUCCESS;
 }
 
 // Operand of D = A * B^T as the GEMM engine reads it.
