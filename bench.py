@@ -33,6 +33,9 @@ WORKLOADS = {
     "bigvocab_fwd_bwd": ("bigvocab_fwd_bwd", "fwd_bwd", {"targets": "zipf"}, 1.0),
     # head-only fine-tuning as in the paper: shared unembedding and trunk frozen (no dE, no dh)
     "finetune_fwd_bwd": ("train_fwd_bwd", "fwd_bwd", {}, None),
+    # the paper's fine-tuning objective (Eq. 14): KL to the frozen head's logits + discounted CE, head only
+    "distill_fwd_bwd": ("train_fwd_bwd", "distill", {}, None),
+    "distill_fwd_bwd_small": ("train_fwd_bwd_small", "distill", {}, None),
     "decode_1": ("decode_1", "score", {}, None),
     "decode_8": ("decode_8", "score", {}, None),
     "decode_64": ("decode_64", "score", {}, None),
@@ -107,6 +110,9 @@ def flops_per_position(s, kind, skip=()):
     fwd = 2 * K * (s.d * s.d + s.V * s.d) + 2 * s.r * s.d
     if kind == "full_fwd_bwd":
         return 3 * (2 * K * s.V * s.d + 2 * s.r * s.d)
+    if kind == "distill":
+        # projection, two vocabulary sweeps forward (log-sum-exp, KL), logits recompute + dz backward, dW_head
+        return 4 * K * s.d * s.d + 4 * 2 * K * s.V * s.d + 2 * s.r * s.d
     if kind == "fwd_bwd" and skip:
         # forward + dz always; dE, dW_head, dh only when asked for
         total = fwd + 2 * K * s.V * s.d
@@ -127,7 +133,13 @@ def oracle_seconds_per_position(inp, kind, aux, sample: int):
     sample = min(sample, s.N)
     sub = synth.subsample_positions(inp, torch.arange(sample))
     t0 = time.perf_counter()
-    if kind == "full_fwd_bwd":
+    if kind == "distill":
+        from oracle import distill
+
+        T = synth.make_teacher_logits(sub.shape, sub.x, seed=0)
+        t0 = time.perf_counter()
+        distill.backward(sub.h, sub.W_head, sub.E, sub.W_g, sub.x, T, s.n, s.r, beta=0.9, gamma=0.8)
+    elif kind == "full_fwd_bwd":
         cp_head.backward_full(sub.h, synth.make_full_head(s, seed=0), sub.W_g, sub.x, s.n, s.r, aux_coef=aux or 0.0)
     elif kind == "fwd_bwd":
         cp_head.backward(sub.h, sub.W_head, sub.E, sub.W_g, sub.x, s.n, s.r, aux_coef=aux or 0.0)
@@ -150,7 +162,7 @@ def blas_threads() -> int:
 
 def oracle_sample_size(s, kind) -> int:
     # about 10-30 s of fp64 numpy work: assume ~40 GFLOP/s on the host cores
-    per_pos = flops_per_position(s, kind) * (1.4 if kind == "fwd_bwd" else 1.0)
+    per_pos = flops_per_position(s, kind) * (1.4 if kind in ("fwd_bwd", "distill") else 1.0)
     return max(1, min(s.N, int(40e9 * 15 / per_pos)))
 
 
@@ -205,8 +217,14 @@ def run_ours(args, rank: int, world: int, local_rank: int):
     ws_fwd = binding.alloc_workspace(binding.workspace_bytes(cs, binding.OP_FORWARD) +
                                      binding.host_staging_bytes(cs) + 512)
     status = torch.zeros(1, dtype=torch.int32, device="cuda")
-    saved = binding.Saved.alloc(cs) if kind == "fwd_bwd" else None
+    saved = binding.Saved.alloc(cs) if kind in ("fwd_bwd", "distill") else None
     W_full = ws_ff = ws_fb = None
+    teacher = dsaved = ws_df = ws_db = None
+    if kind == "distill":
+        teacher = synth.make_teacher_logits(shape, inp.x, seed=dist_util.shard_seed(0, rank)).cuda()
+        dsaved = binding.DistillSaved.alloc(cs)
+        ws_df = binding.alloc_workspace(binding.workspace_bytes(cs, binding.OP_DISTILL_FORWARD))
+        ws_db = binding.alloc_workspace(binding.workspace_bytes(cs, binding.OP_DISTILL_BACKWARD))
     if kind == "full_fwd_bwd":
         W_full = synth.make_full_head(shape, seed=dist_util.shard_seed(0, rank)).cuda()
         saved = binding.Saved.alloc_full(cs)
@@ -215,7 +233,7 @@ def run_ours(args, rank: int, world: int, local_rank: int):
     ws_bwd = binding.alloc_workspace(binding.workspace_bytes(cs, binding.OP_BACKWARD)) if kind == "fwd_bwd" else None
     ws_smp = binding.alloc_workspace(binding.workspace_bytes(cs, binding.OP_SAMPLE)) if kind == "sample" else None
     out_f, out_b, out_s = {}, {}, {}
-    skip = ("dE", "dh") if args.workload == "finetune_fwd_bwd" else ()
+    skip = ("dE", "dh") if args.workload == "finetune_fwd_bwd" or kind == "distill" else ()
 
     def step():
         if kind == "fwd":
@@ -225,6 +243,11 @@ def run_ours(args, rank: int, world: int, local_rank: int):
                             out=out_f)
             binding.backward(h, W_head, E, W_g, x, saved, aux_coef=aux, workspace=ws_bwd, dev_status=status,
                              out=out_b, skip=skip)
+        elif kind == "distill":
+            binding.distill_forward(h, W_head, E, W_g, x, teacher, saved, dsaved, beta=0.9, gamma=0.8,
+                                    workspace=ws_df, dev_status=status, out=out_f)
+            binding.distill_backward(h, W_head, E, W_g, x, teacher, saved, dsaved, beta=0.9, gamma=0.8,
+                                     workspace=ws_db, dev_status=status, out=out_b, skip=skip)
         elif kind == "sample":
             binding.sample_draft(h, W_head, E, W_g, shape.n, topk=5, workspace=ws_smp, dev_status=status, out=out_s)
         elif kind == "full_fwd_bwd":
@@ -246,7 +269,7 @@ def run_ours(args, rank: int, world: int, local_rank: int):
             draft_pin.copy_(out_s["draft"], non_blocking=True)
             torch.cuda.current_stream().synchronize()
             return
-        if kind == "full_fwd_bwd":
+        if kind in ("full_fwd_bwd", "distill"):
             h.copy_(h_pin, non_blocking=True)
             x.copy_(x_pin, non_blocking=True)
             step()
@@ -299,7 +322,7 @@ def run_ours(args, rank: int, world: int, local_rank: int):
     value = dist_util.whole_job_rate(shape.N, args.steps, world, ms_total)
     e2e_value = dist_util.whole_job_rate(shape.N, args.steps, world, ms_e2e)
     K = shape.n * shape.r
-    dominant = "lse"
+    dominant = "kl" if kind == "distill" else "lse"
     dom_ms, dom_launches = stages.get(dominant, (0.0, 0))
     avg_ms = dom_ms / max(1, dom_launches)
     if kind in ("score", "sample") and shape.N * K * 2 < 250:   # below the ridge: HBM-bound streaming of E
@@ -314,6 +337,8 @@ def run_ours(args, rank: int, world: int, local_rank: int):
     roof["frac"] = roof["achieved"] / roof["peak"]
     roof["traffic"] = NCU_TRAFFIC_BYTES.get(args.workload)
     roof["kernel"] = "tc_gemm_kernel<EpiLse> (unembedding + logsumexp_V)"
+    if kind == "distill":
+        roof["kernel"] = "tc_gemm_kernel<EpiKl> (unembedding + expert mixture + KL to the teacher, grouped rows)"
     if kind == "full_fwd_bwd":
         roof["kernel"] = "tc_gemm_kernel<EpiLseFull> (all heads' unembeddings + logsumexp_V in one GEMM)"
     roof["peak_source"] = peaks["src"]

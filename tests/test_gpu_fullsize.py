@@ -211,3 +211,42 @@ def test_bigvocab_full_size_forward_and_backward_sampled():
     up = np.full(len(idx), -1.0 / s.N)
     ref = cp_head.backward(sub.h, sub.W_head, sub.E, sub.W_g, sub.x, s.n, s.r, dloss_dlogp=up)
     assert rel_l2(g0["dh"][idx.cuda()].float().cpu().numpy(), ref.dh) <= GRAD_TOL
+
+
+def test_distill_full_size_sampled_kl_and_dh():
+    """Eq. 14 at the fine-tuning size the benchmark times (N = 8192, d = 4096, V = 32000, n = 4, r = 8):
+    KL terms, prefix scores and dh on sampled positions against the oracle run on just those positions
+    with the full batch's weights; the loss against a host sum of the device's own per-position terms."""
+    from oracle import distill
+    from paper_2410_17765_b200 import binding
+
+    inp = inputs_for("train_fwd_bwd")
+    s = inp.shape
+    T = synth.make_teacher_logits(s, inp.x, seed=0)
+    dev = to_dev(inp) + [T.cuda()]
+    cs = binding.make_shape(s.N, s.d, s.V, s.n, s.r)
+    saved, dsaved = binding.Saved.alloc(cs), binding.DistillSaved.alloc(cs)
+    st = torch.zeros(1, dtype=torch.int32, device="cuda")
+    beta, gamma = 0.9, 0.8
+    out = binding.distill_forward(*dev, saved, dsaved, beta=beta, gamma=gamma, dev_status=st)
+    g = binding.distill_backward(*dev, saved, dsaved, beta=beta, gamma=gamma, dev_status=st, skip=("dE",))
+    torch.cuda.synchronize()
+    assert int(st.item()) == 0
+    kl = out["kl"].cpu().numpy()
+    prefix = out["logp_prefix"].cpu().numpy()
+    assert np.all(np.isfinite(kl)) and np.all(kl > -1e-4)
+    idx = sample_positions(s.N, 6, seed=3)
+    sub = synth.subsample_positions(inp, idx)
+    Tsub = T[idx]
+    ref = distill.forward(sub.h, sub.W_head, sub.E, sub.W_g, sub.x, Tsub, s.n, s.r, beta=beta, gamma=gamma)
+    assert np.max(np.abs(kl[idx.numpy()] - ref.kl)) <= LOGP_TOL
+    assert np.max(np.abs(prefix[idx.numpy()] - ref.prefix)) <= LOGP_TOL
+    disc = gamma ** np.arange(s.n)
+    ce = -np.diff(np.concatenate([np.zeros((s.N, 1)), prefix.astype(np.float64)], axis=1), axis=1)
+    want = float(np.sum(disc * (beta * kl.astype(np.float64) + (1 - beta) * ce)) / s.N)
+    assert abs(float(out["loss"].item()) - want) <= 1e-4
+    # dh of a position depends on that position only: oracle on the sample with the full batch's 1/N weights
+    up, uk = distill.loss_weights(s.N, s.n, beta, gamma)
+    gr = distill.backward(sub.h, sub.W_head, sub.E, sub.W_g, sub.x, Tsub, s.n, s.r, dloss_dprefix=up[: len(idx)],
+                          dloss_dkl=uk[: len(idx)])
+    assert rel_l2(g["dh"][idx.cuda()].float().cpu().numpy(), gr.dh) <= GRAD_TOL
