@@ -36,6 +36,7 @@ CASES = {
     # d = 4096: the logits carry the bf16 rounding of z (2^-9 relative on sums of 4096 terms), which a KL over
     # only 600 tokens does not average out; paper-like weight scale, and see the test for the two bounds
     "long_k": dict(shape=synth.Shape(N=40, d=4096, V=600, n=2, r=8), weight_scale=1.0),
+    "long_k_rank3": dict(shape=synth.Shape(N=100, d=4096, V=520, n=2, r=3), weight_scale=1.0),   # long contraction with padded groups
 }
 
 
@@ -77,11 +78,13 @@ def test_distill_forward_and_backward_match_oracle(name):
     inp, T, s, out, g, dsaved = run_case(name, aux=0.5)
     ref = distill.forward(inp.h, inp.W_head, inp.E, inp.W_g, inp.x, T, s.n, s.r, beta=0.9, gamma=0.8, aux_coef=0.5)
     kl = out["kl"].cpu().numpy()
-    if name == "long_k":
-        # against the oracle's bf16-z mode the bar holds; the exact mode differs by z's rounding itself
+    if name.startswith("long_k"):
+        # against the oracle's bf16-z mode the bar holds; the exact mode differs by z's rounding itself: a KL
+        # weighs the perturbed probabilities by log-ratios of size ~10, so the logit rounding that moves a
+        # log-sum-exp by up to 2e-3 at these shapes moves a KL over ~500 tokens by up to ~1e-2
         contract = distill.forward(inp.h, inp.W_head, inp.E, inp.W_g, inp.x, T, s.n, s.r, round_z=True)
         assert np.max(np.abs(kl - contract.kl)) <= TOL
-        assert np.max(np.abs(kl - ref.kl)) <= 3 * TOL
+        assert np.max(np.abs(kl - ref.kl)) <= 10 * TOL
     else:
         assert np.max(np.abs(kl - ref.kl)) <= TOL
     assert np.max(np.abs(out["logp_prefix"].cpu().numpy() - ref.prefix)) <= TOL
