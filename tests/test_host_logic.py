@@ -68,3 +68,26 @@ def test_null_and_misaligned_pointers_are_rejected(lib):
     assert lib.cpmtp_forward(ctypes.byref(s), odd, p, p, p, p, p, None, None, None, p, 4096, None, None) == -3
     assert lib.cpmtp_backward(ctypes.byref(s), p, p, p, p, p, None, None, p, p, p, p, p, 4096, None, None) in (-1, -5, -6)
     assert lib.cpmtp_forward(None, p, p, p, p, p, p, None, None, None, p, 4096, None, None) == -1
+
+
+def test_distill_workspace_and_argument_checks(lib):
+    s = binding.make_shape(64, 256, 1024, 3, 3)
+    fwd = binding.workspace_bytes(s, binding.OP_FORWARD)
+    dfwd = binding.workspace_bytes(s, binding.OP_DISTILL_FORWARD)
+    dbwd = binding.workspace_bytes(s, binding.OP_DISTILL_BACKWARD)
+    assert dfwd > fwd                                   # the plain forward plus the KL partials
+    # backward: dz, one chunk of logit gradients of whole padded tiles (32 groups of 3 rows), weights per (i, k)
+    assert dbwd >= 2 * 64 * 9 * 256 + 2 * 96 * 1024 + 4 * 64 * 3
+    buf = (ctypes.c_char * 8192)()
+    base = ctypes.addressof(buf)
+    base += (-base) % 256
+    p = ctypes.c_void_p(base)
+    f = ctypes.c_float
+    # shape errors come first, then missing pointers
+    bad = binding.make_shape(64, 100, 1024, 3, 3)
+    assert lib.cpmtp_distill_forward(ctypes.byref(bad), p, p, p, p, p, p, f(0.9), f(1.0), p, p, None, None, None,
+                                     p, 4096, None, None) == -2
+    assert lib.cpmtp_distill_forward(ctypes.byref(s), p, p, p, p, p, None, f(0.9), f(1.0), p, p, None, None, None,
+                                     p, 4096, None, None) in (-1, -5, -6)
+    assert lib.cpmtp_distill_backward(ctypes.byref(s), p, p, p, p, p, None, None, None, f(0.9), f(1.0), None, None,
+                                      p, p, p, p, p, 4096, None, None) == -1
