@@ -75,3 +75,62 @@ def test_random_shape(it):
     for key, want in (("dh", reffg.dh), ("dW_full", reffg.dW_full), ("dW_g", reffg.dW_g)):
         if np.linalg.norm(want) > 0:
             assert rel_l2(gf[key].float().cpu().numpy(), want) <= 1e-2, (shape, key)
+
+
+def random_distill_case(it):
+    rng = np.random.default_rng(5000 + it)
+    d = int(rng.choice([64, 128, 192, 256, 512, 1024]))
+    n = int(rng.integers(1, 5))
+    r = int(rng.choice([1, 2, 3, 4, 5, 6, 7, 8, 12, 16, 32]))
+    N = int(rng.choice([1, 2, 7, 33, 128, 129, 300]))
+    V = int(rng.integers(2, 2500))
+    if rng.random() < 0.4:
+        V = (V + 7) // 8 * 8          # vector teacher loads
+    cost = n * r * (d * d + V * d)
+    if N * cost > 8e9:
+        N = max(1, int(8e9 / cost))
+    mem = N * n * r * V * 8 * 3       # the oracle keeps [N, n, r, V] fp64 arrays
+    if mem > 2e9:
+        N = max(1, int(N * 2e9 / mem))
+    return synth.Shape(N, d, V, n, r), float(rng.choice([0.0, 0.5, 0.9, 1.0])), float(rng.choice([0.7, 1.0])), \
+        float(rng.choice([0.0, 1.0])), int(rng.choice([0, 96, 256, 1024]))
+
+
+@pytest.mark.parametrize("it", range(10))
+def test_random_distill_shape(it):
+    """Eq. 14 on random shapes: every padded-rank instantiation, ragged groups and vocabularies, both teacher
+    load paths, chunked backward."""
+    from oracle import distill
+    from paper_2410_17765_b200 import binding
+
+    shape, beta, gamma, aux, chunk = random_distill_case(it)
+    n, r = shape.n, shape.r
+    inp = synth.make_inputs(shape, seed=100 + it, weight_scale=2.0 if shape.d <= 512 else 1.0)
+    T = synth.make_teacher_logits(shape, inp.x, seed=it)
+    ref = distill.forward(inp.h, inp.W_head, inp.E, inp.W_g, inp.x, T, n, r, beta=beta, gamma=gamma, aux_coef=aux)
+    refg = distill.backward(inp.h, inp.W_head, inp.E, inp.W_g, inp.x, T, n, r, beta=beta, gamma=gamma, aux_coef=aux)
+    dev = [t.cuda() for t in (inp.h, inp.W_head, inp.E, inp.W_g, inp.x, T)]
+    cs = binding.make_shape(shape.N, shape.d, shape.V, n, r)
+    st = torch.zeros(1, dtype=torch.int32, device="cuda")
+    saved, dsaved = binding.Saved.alloc(cs), binding.DistillSaved.alloc(cs)
+    old = os.environ.get("CPMTP_BWD_CHUNK_ROWS")
+    try:
+        if chunk:
+            os.environ["CPMTP_BWD_CHUNK_ROWS"] = str(chunk)
+        out = binding.distill_forward(*dev, saved, dsaved, beta=beta, gamma=gamma, aux_coef=aux if aux else None,
+                                      dev_status=st)
+        g = binding.distill_backward(*dev, saved, dsaved, beta=beta, gamma=gamma, aux_coef=aux if aux else None,
+                                     dev_status=st)
+        torch.cuda.synchronize()
+    finally:
+        if old is None:
+            os.environ.pop("CPMTP_BWD_CHUNK_ROWS", None)
+        else:
+            os.environ["CPMTP_BWD_CHUNK_ROWS"] = old
+    assert int(st.item()) == 0, shape
+    assert np.abs(out["kl"].cpu().numpy() - ref.kl).max() <= 2e-3, shape
+    assert np.abs(out["logp_prefix"].cpu().numpy() - ref.prefix).max() <= 2e-3, shape
+    assert abs(float(out["loss"].item()) - ref.loss) <= 2e-3, shape
+    for key, want in (("dh", refg.dh), ("dW_head", refg.dW_head), ("dE", refg.dE), ("dW_g", refg.dW_g)):
+        if np.linalg.norm(want) > 0:
+            assert rel_l2(g[key].float().cpu().numpy(), want) <= 1e-2, (shape, key)
