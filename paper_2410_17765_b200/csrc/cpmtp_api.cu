@@ -539,57 +539,17 @@ static int sms_or_default() {
 
 
 // The two grouped passes, instantiated for every padded rank R (a power of two, 1..32).
-template <int RR>
-static cudaError_t distill_kl_r(const uint16_t* z, long long rows, int d, const uint16_t* E, int V, const Sched& sc,
-                                float* part, const float* lse, const float* logpi, const float* lse_t,
-                                const uint16_t* T, int groups, int r, int* dev_status, int sms, cudaStream_t st) {
-  typename EpiKl<kBN, RR>::Params ep{part, lse, logpi, lse_t, T, groups, r, V, sc.n_splits, V % 8 == 0 ? 1 : 0};
-  return launch_gemm<CfgKK, EpiKl<kBN, RR>>(z, rows, d, E, V, d, d, sc, ep, dev_status, sms, st, r);
-}
-
-static cudaError_t launch_distill_kl(int R, const uint16_t* z, long long rows, int d, const uint16_t* E, int V,
-                                     const Sched& sc, float* part, const float* lse, const float* logpi,
-                                     const float* lse_t, const uint16_t* T, int groups, int r, int* dev_status,
-                                     int sms, cudaStream_t st) {
-  switch (R) {
-    case 1: return distill_kl_r<1>(z, rows, d, E, V, sc, part, lse, logpi, lse_t, T, groups, r, dev_status, sms, st);
-    case 2: return distill_kl_r<2>(z, rows, d, E, V, sc, part, lse, logpi, lse_t, T, groups, r, dev_status, sms, st);
-    case 4: return distill_kl_r<4>(z, rows, d, E, V, sc, part, lse, logpi, lse_t, T, groups, r, dev_status, sms, st);
-    case 8: return distill_kl_r<8>(z, rows, d, E, V, sc, part, lse, logpi, lse_t, T, groups, r, dev_status, sms, st);
-    case 16: return distill_kl_r<16>(z, rows, d, E, V, sc, part, lse, logpi, lse_t, T, groups, r, dev_status, sms, st);
-    case 32: return distill_kl_r<32>(z, rows, d, E, V, sc, part, lse, logpi, lse_t, T, groups, r, dev_status, sms, st);
-    default: return cudaErrorInvalidValue;
-  }
-}
-
-template <int RR>
-static cudaError_t distill_grad_r(const uint16_t* z, long long rows, int d, const uint16_t* E, const Sched& sc,
-                                  const typename EpiDistillGrad<kBN, RR>::Params& ep, int r, int* dev_status, int sms,
+template <template <int, int> class Epi, class Params>
+static cudaError_t launch_grouped(int R, const uint16_t* z, long long rows, int d, const uint16_t* E, int V,
+                                  const Sched& sc, const Params& ep, int r, int* dev_status, int sms,
                                   cudaStream_t st) {
-  // the column tiles that cover V also cover the padding columns [V, ldg), which are written as zero
-  return launch_gemm<CfgKK, EpiDistillGrad<kBN, RR>>(z, rows, d, E, ep.V, d, d, sc, ep, dev_status, sms, st, r);
-}
-
-static cudaError_t launch_distill_grad(int R, const uint16_t* z, long long rows, int d, const uint16_t* E, int V,
-                                       const Sched& sc, uint16_t* G, const cpmtp_saved* saved, const float* coef,
-                                       const cpmtp_distill_saved* ds, const float* uk, const uint16_t* T,
-                                       const int32_t* x, long long grp0, int groups, int r, int ldg,
-                                       int* dev_status, int sms, cudaStream_t st) {
-  // identical parameter blocks for every R
-  const EpiDistillGrad<kBN, 1>::Params p1{G, saved->lse, coef, ds->logpi, ds->pm, uk, ds->lse_t, T, x,
-                                          grp0, groups, r, V, ldg, V % 8 == 0 ? 1 : 0};
-  auto as = [&](auto tag) {
-    typename decltype(tag)::Params q{p1.G, p1.lse, p1.coef, p1.logpi, p1.pm, p1.uk, p1.lse_t, p1.T, p1.x,
-                                     p1.grp0, p1.groups, p1.r, p1.V, p1.ldg, p1.vec};
-    return q;
-  };
   switch (R) {
-    case 1: return distill_grad_r<1>(z, rows, d, E, sc, as(EpiDistillGrad<kBN, 1>{}), r, dev_status, sms, st);
-    case 2: return distill_grad_r<2>(z, rows, d, E, sc, as(EpiDistillGrad<kBN, 2>{}), r, dev_status, sms, st);
-    case 4: return distill_grad_r<4>(z, rows, d, E, sc, as(EpiDistillGrad<kBN, 4>{}), r, dev_status, sms, st);
-    case 8: return distill_grad_r<8>(z, rows, d, E, sc, as(EpiDistillGrad<kBN, 8>{}), r, dev_status, sms, st);
-    case 16: return distill_grad_r<16>(z, rows, d, E, sc, as(EpiDistillGrad<kBN, 16>{}), r, dev_status, sms, st);
-    case 32: return distill_grad_r<32>(z, rows, d, E, sc, as(EpiDistillGrad<kBN, 32>{}), r, dev_status, sms, st);
+    case 1: return launch_gemm<CfgKK, Epi<kBN, 1>>(z, rows, d, E, V, d, d, sc, ep, dev_status, sms, st, r);
+    case 2: return launch_gemm<CfgKK, Epi<kBN, 2>>(z, rows, d, E, V, d, d, sc, ep, dev_status, sms, st, r);
+    case 4: return launch_gemm<CfgKK, Epi<kBN, 4>>(z, rows, d, E, V, d, d, sc, ep, dev_status, sms, st, r);
+    case 8: return launch_gemm<CfgKK, Epi<kBN, 8>>(z, rows, d, E, V, d, d, sc, ep, dev_status, sms, st, r);
+    case 16: return launch_gemm<CfgKK, Epi<kBN, 16>>(z, rows, d, E, V, d, d, sc, ep, dev_status, sms, st, r);
+    case 32: return launch_gemm<CfgKK, Epi<kBN, 32>>(z, rows, d, E, V, d, d, sc, ep, dev_status, sms, st, r);
     default: return cudaErrorInvalidValue;
   }
 }
@@ -670,8 +630,10 @@ static int backward_impl(const cpmtp_shape* shape, const void* h, const void* W_
       const int groups = rows / s.r;   // chunks hold whole groups
       Sched sc = make_sched((groups + gpt - 1) / gpt, (V + kBN - 1) / kBN, (V + kBN - 1) / kBN, 2048 / kBM, d / kBK);
       sc.a_groups = gpt;
-      CPMTP_TRY(launch_distill_grad(R, zc, rows, d, Eb, V, sc, G, saved, coef, dc->ds, uk, dc->teacher, x,
-                                    row0 / s.r, groups, s.r, L.ldg, dev_status, sms, st));
+      // the column tiles that cover V also cover the padding columns [V, ldg), which are written as zero
+      const DistillGradParams ep{G, saved->lse, coef, dc->ds->logpi, dc->ds->pm, uk, dc->ds->lse_t, dc->teacher, x,
+                                 row0 / s.r, groups, s.r, V, L.ldg, V % 8 == 0 ? 1 : 0};
+      CPMTP_TRY((launch_grouped<EpiDistillGrad>(R, zc, rows, d, Eb, V, sc, ep, s.r, dev_status, sms, st)));
     } else if (need_dz || dE != nullptr) {
       ProfScope prof(CPMTP_STAGE_LOGIT_GRAD, st);
       EpiLogitGrad<kBN>::Params ep{G, saved->lse, coef, x, row0, rows, L.ldg, V, K, s.n, s.r};
@@ -1121,8 +1083,10 @@ int cpmtp_distill_forward(const cpmtp_shape* shape, const void* h, const void* W
   float* part = reinterpret_cast<float*>(ws + L.part);
   {
     ProfScope prof(CPMTP_STAGE_KL, st);
-    CPMTP_TRY(launch_distill_kl(L.R, z, L.fwd.M, s.d, static_cast<const uint16_t*>(E), s.V, L.sched, part, saved->lse,
-                                dsaved->logpi, dsaved->lse_t, Tb, L.groups, s.r, dev_status, di->sms, st));
+    const KlParams ep{part, saved->lse, dsaved->logpi, dsaved->lse_t, Tb, L.groups, s.r, s.V, L.sched.n_splits,
+                      s.V % 8 == 0 ? 1 : 0};
+    CPMTP_TRY((launch_grouped<EpiKl>(L.R, z, L.fwd.M, s.d, static_cast<const uint16_t*>(E), s.V, L.sched, ep, s.r,
+                                     dev_status, di->sms, st)));
   }
   {
     ProfScope prof(CPMTP_STAGE_FINALIZE, st);

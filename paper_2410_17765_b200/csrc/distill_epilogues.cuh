@@ -103,16 +103,18 @@ __device__ __forceinline__ void finish_columns(float* pd, const uint16_t* __rest
 // ---------------------------------------------------------------------------
 // Forward: pm[(g, a)] = sum_v e(v) l(v) with e = pi_{g,a} P^(k)(v | a); the KL term of Eq. 14 for
 // group g is sum_a pm[(g, a)].  One partial per (row, split); rows are ORIGINAL rows g * r + a.
+struct KlParams {
+  float* part;            // [groups * r, splits]
+  const float* lse;       // [groups * r]  logsumexp_v S
+  const float* logpi;     // [groups * r]  log pi
+  const float* lse_t;     // [groups]      logsumexp_v T
+  const uint16_t* T;      // [groups, V]   teacher logits, bf16
+  int groups, r, V, splits, vec;
+};
+
 template <int BN, int R>
 struct EpiKl {
-  struct Params {
-    float* part;            // [groups * r, splits]
-    const float* lse;       // [groups * r]  logsumexp_v S
-    const float* logpi;     // [groups * r]  log pi
-    const float* lse_t;     // [groups]      logsumexp_v T
-    const uint16_t* T;      // [groups, V]   teacher logits, bf16
-    int groups, r, V, splits, vec;
-  };
+  using Params = KlParams;
   struct State { float c2, lt, acc; long long orow; int grp; bool valid, grp_ok; };
   static constexpr int SMEM_BYTES = 0;
   using GL = GroupLanes<R>;
@@ -164,21 +166,23 @@ struct EpiKl {
 // Backward: logit gradient of  sum up * prefix + sum uk * kl  for a chunk of groups,
 //   G[(g,a), v] = coef (1[v = x_g] - P(v)) + uk_g (e(v) l(v) - P(v) pm[(g,a)]),
 // bf16, written at ORIGINAL rows relative to the chunk.  Columns in [V, ldg) are zero.
+struct DistillGradParams {
+  uint16_t* G;            // [groups * r, ldg] bf16 (this chunk)
+  const float* lse;       // the arrays below are indexed by GLOBAL row / group
+  const float* coef;      // [.., r]  d objective / d C  (cross-entropy and KL-weight paths)
+  const float* logpi;
+  const float* pm;
+  const float* uk;        // [groups_total]
+  const float* lse_t;     // [groups_total]
+  const uint16_t* T;      // [groups_total, V]
+  const int32_t* x;       // [groups_total]
+  long long grp0;         // first group of the chunk
+  int groups, r, V, ldg, vec;
+};
+
 template <int BN, int R>
 struct EpiDistillGrad {
-  struct Params {
-    uint16_t* G;            // [groups * r, ldg] bf16 (this chunk)
-    const float* lse;       // the arrays below are indexed by GLOBAL row / group
-    const float* coef;      // [.., r]  d objective / d C  (cross-entropy and KL-weight paths)
-    const float* logpi;
-    const float* pm;
-    const float* uk;        // [groups_total]
-    const float* lse_t;     // [groups_total]
-    const uint16_t* T;      // [groups_total, V]
-    const int32_t* x;       // [groups_total]
-    long long grp0;         // first group of the chunk
-    int groups, r, V, ldg, vec;
-  };
+  using Params = DistillGradParams;
   struct State { float lse2, pi, coef, ukpi, ckm, lt; long long grp, orow_local; int tok; bool valid, grp_ok; };
   static constexpr int SMEM_BYTES = 0;
   using GL = GroupLanes<R>;
