@@ -625,7 +625,7 @@ static int backward_impl(const cpmtp_shape* shape, const void* h, const void* W_
     const int rows = static_cast<int>((L.M - row0) < L.chunk_rows ? (L.M - row0) : L.chunk_rows);
     const uint16_t* zc = z + row0 * d;
     // recompute logits tile by tile -> G = dloss/dS (bf16), never more than one chunk
-    if (dc != nullptr) {
+    if (dc != nullptr && (need_dz || dE != nullptr)) {
       ProfScope prof(CPMTP_STAGE_LOGIT_GRAD, st);
       const int groups = rows / s.r;   // chunks hold whole groups
       Sched sc = make_sched((groups + gpt - 1) / gpt, (V + kBN - 1) / kBN, (V + kBN - 1) / kBN, 2048 / kBM, d / kBK);
@@ -634,7 +634,7 @@ static int backward_impl(const cpmtp_shape* shape, const void* h, const void* W_
       const DistillGradParams ep{G, saved->lse, coef, dc->ds->logpi, dc->ds->pm, uk, dc->ds->lse_t, dc->teacher, x,
                                  row0 / s.r, groups, s.r, V, L.ldg, V % 8 == 0 ? 1 : 0};
       CPMTP_TRY((launch_grouped<EpiDistillGrad>(R, zc, rows, d, Eb, V, sc, ep, s.r, dev_status, sms, st)));
-    } else if (need_dz || dE != nullptr) {
+    } else if (dc == nullptr && (need_dz || dE != nullptr)) {
       ProfScope prof(CPMTP_STAGE_LOGIT_GRAD, st);
       EpiLogitGrad<kBN>::Params ep{G, saved->lse, coef, x, row0, rows, L.ldg, V, K, s.n, s.r};
       CPMTP_TRY((gemm_auto<false, false, EpiLogitGrad<kBN>>(zc, d, Eb, d, rows, V, d, 2048, ep, dev_status, sms, st)));
