@@ -308,6 +308,16 @@ def run_ours(args, rank: int, world: int, local_rank: int):
     sampler = ClockSampler(local_rank) if rank == 0 else None
     ms_total, stages = timed(step, args.steps, True)
     clocks = sampler.stop() if sampler is not None else None
+    graph_ms = None
+    if kind == "score":   # launch-bound regime: the same step replayed from a CUDA graph
+        side = torch.cuda.Stream()
+        side.wait_stream(torch.cuda.current_stream())
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph, stream=side):
+            step()
+        for _ in range(3):
+            graph.replay()
+        graph_ms, _ = timed(graph.replay, args.steps, False)
     for _ in range(min(args.warmup, 3)):
         step_e2e()
     ms_e2e, _ = timed(step_e2e, args.steps, False)
@@ -366,6 +376,8 @@ def run_ours(args, rank: int, world: int, local_rank: int):
         "model_flops_tflops": total_flops / (ms_total * 1e-3) / 1e12,
         "stages_ms_per_step": {k: v[0] / args.steps for k, v in stages.items()},
     }
+    if graph_ms is not None:
+        line["cuda_graph_ms_per_step"] = graph_ms / args.steps
     print(json.dumps(line))
     dist_util.finalize()
 

@@ -28,6 +28,9 @@
  *    expired (results invalid).
  *  - Limits: d % 64 == 0, 1 <= r <= 32, 1 <= n <= 8, N >= 1, V >= 2,
  *    N*n*r*d < 2^40.
+ *  - CUDA graphs: the entry points only enqueue kernels and copies, so they may be recorded by stream
+ *    capture and replayed (same pointers, new contents); call each once outside capture first, since the
+ *    first launch of a kernel sets its shared-memory attribute.  Environment knobs are read at capture time.
  *  - Threads: calls may be made from several host threads as long as each uses
  *    its own stream, workspace and outputs; the per-stage profiling calls are
  *    the exception (one thread, one device).
