@@ -49,8 +49,8 @@ WORKLOADS = {
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel, from the ncu
 # captures summarised under profiles/ (None until captured, or once the kernel has changed since).
 NCU_TRAFFIC_BYTES = {
-    "train_fwd": 1.236112e9 + 5.9648e6,   # profiles/lse_train_fwd.md
-    "decode_1": 1.05168e9 + 3.763968e6,    # profiles/decode_1.md
+    "train_fwd": 1.211966e9 + 5.231616e6,   # profiles/lse_train_fwd.md
+    "decode_1": 1.051677e9 + 3.764992e6,    # profiles/decode_1.md
 }
 
 
@@ -309,7 +309,7 @@ def run_ours(args, rank: int, world: int, local_rank: int):
     ms_total, stages = timed(step, args.steps, True)
     clocks = sampler.stop() if sampler is not None else None
     graph_ms = None
-    if kind == "score":   # launch-bound regime: the same step replayed from a CUDA graph
+    if kind == "score" and not args.no_graph:   # launch-bound regime: the same step replayed from a CUDA graph
         side = torch.cuda.Stream()
         side.wait_stream(torch.cuda.current_stream())
         graph = torch.cuda.CUDAGraph()
@@ -389,6 +389,7 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="train_fwd", choices=sorted(WORKLOADS))
+    ap.add_argument("--no-graph", action="store_true", help="skip the CUDA-graph replay leg of the decode workloads")
     args = ap.parse_args()
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
