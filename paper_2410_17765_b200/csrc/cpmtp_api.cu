@@ -236,6 +236,23 @@ DistillLayout distill_layout(const cpmtp_shape& s, int sms) {
   const int m_tiles = (L.groups + L.gpt - 1) / L.gpt;
   const int n_tiles = (s.V + kBN - 1) / kBN;
   L.sched = sched_lse(m_tiles, n_tiles, m_tiles * kBM, s.V, s.d, kBM, sms);
+  if (s.d >= 4096 && m_tiles >= 16) {
+    // Long contractions: short units in the raster of the plain GEMMs (16 row tiles x up to 125 vocabulary
+    // ranges) beat the long lock-stepped sweeps, as for the 256-row unembedding: measured 54.2 ms against
+    // 57.6 ms at N = 8192, d = 4096, V = 32000, n = 4, r = 8 (interleaved A/B in one process); at d = 2048 the
+    // sweeps of sched_lse stay ahead (6.8 ms against 7.2 ms at N = 4096, V = 32000, n = 2, r = 8).
+    int sp = n_tiles < 125 ? n_tiles : 125;
+    if ((16ll * sp) % sms == 0 && sp > 1) --sp;
+    L.sched = make_sched(m_tiles, n_tiles, sp, 16, s.d / kBK);
+  }
+  {
+    // tuning knobs for this sweep alone
+    int g = 0, sp = 0;
+    if (const char* env = std::getenv("CPMTP_KL_GROUP_TILES")) g = std::atoi(env);
+    if (const char* env = std::getenv("CPMTP_KL_SPLITS")) sp = std::atoi(env);
+    if (g >= 1 || sp >= 1)
+      L.sched = make_sched(m_tiles, n_tiles, sp >= 1 ? sp : L.sched.n_splits, g >= 1 ? g : L.sched.m_group, s.d / kBK);
+  }
   L.sched.a_groups = L.gpt;
   size_t off = align_up(L.fwd.total);
   auto take = [&](size_t bytes) { size_t o = off; off = align_up(off + bytes); return o; };
