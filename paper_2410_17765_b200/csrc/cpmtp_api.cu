@@ -848,7 +848,7 @@ int cpmtp_sample_draft(const cpmtp_shape* shape, const void* h, const void* W_he
     draft_step_partial_kernel<<<dim3(L.chunks, s.N), kSampleThreads, 0, st>>>(
         logits, L.lds, lse, lb, uniform, inv_temp, step, s.V, s.n, s.r, topk, part_top, part_best);
     CPMTP_TRY(cudaGetLastError());
-    draft_step_final_kernel<<<s.N, kSampleThreads, 0, st>>>(z32, static_cast<const uint16_t*>(E), s.d, lse, lb,
+    draft_step_final_kernel<<<s.N, kSampleFinalThreads, 0, st>>>(z32, static_cast<const uint16_t*>(E), s.d, lse, lb,
                                                            part_top, part_best, L.chunks,
                                                            uniform != nullptr ? 1 : 0, step, s.V, s.n, s.r, topk,
                                                            draft, logp_joint, topk_tokens, topk_logp);

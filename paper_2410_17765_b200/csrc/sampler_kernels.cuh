@@ -20,6 +20,7 @@ namespace cpmtp {
 constexpr int kMaxTopk = 8;
 constexpr int kSampleThreads = 256;
 constexpr int kSampleChunk = 2048;   // vocabulary entries per block in the partial pass
+constexpr int kSampleFinalThreads = 1024;   // merge pass: one block per position, one warp per (candidate, expert) dot
 
 struct Cand {
   float score;
@@ -154,7 +155,7 @@ __global__ void draft_step_partial_kernel(const float* __restrict__ S, int lds, 
 // The logits of the drafted token and of the candidates are recomputed from the unrounded z (fp32),
 // as on the likelihood path, so the reported log-probabilities do not carry the bf16 rounding of z
 // (the selection itself is made on the stored logits; candidates keep the selection order).
-__global__ void draft_step_final_kernel(const float* __restrict__ z32, const uint16_t* __restrict__ E, int d,
+__global__ void __launch_bounds__(kSampleFinalThreads) draft_step_final_kernel(const float* __restrict__ z32, const uint16_t* __restrict__ E, int d,
                                         const float* __restrict__ lse,
                                         float* __restrict__ lb, const Cand* __restrict__ part_top,
                                         const Cand* __restrict__ part_best, int chunks, int sampled, int s, int V,
@@ -196,10 +197,23 @@ __global__ void draft_step_final_kernel(const float* __restrict__ z32, const uin
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, nwarps = blockDim.x >> 5;
     for (int job = warp; job < (topk + 1) * r; job += nwarps) {
       const int j = job / r, a = job - j * r;
-      const uint16_t* erow = E + static_cast<size_t>(cand_tok[j]) * d;
-      const float* zrow = z32 + (static_cast<size_t>(i) * K + static_cast<size_t>(s) * r + a) * d;
+      // d % 64 == 0 and 16-byte aligned rows: 8 elements per lane and load
+      const uint4* erow = reinterpret_cast<const uint4*>(E + static_cast<size_t>(cand_tok[j]) * d);
+      const float4* zrow =
+          reinterpret_cast<const float4*>(z32 + (static_cast<size_t>(i) * K + static_cast<size_t>(s) * r + a) * d);
       float acc = 0.f;
-      for (int t = lane; t < d; t += 32) acc = fmaf(__uint_as_float(static_cast<uint32_t>(erow[t]) << 16), zrow[t], acc);
+      for (int t = lane; t < (d >> 3); t += 32) {
+        const uint4 e = __ldg(erow + t);
+        const float4 z0 = zrow[2 * t], z1 = zrow[2 * t + 1];
+        acc = fmaf(ptx::bf16_lo(e.x), z0.x, acc);
+        acc = fmaf(ptx::bf16_hi(e.x), z0.y, acc);
+        acc = fmaf(ptx::bf16_lo(e.y), z0.z, acc);
+        acc = fmaf(ptx::bf16_hi(e.y), z0.w, acc);
+        acc = fmaf(ptx::bf16_lo(e.z), z1.x, acc);
+        acc = fmaf(ptx::bf16_hi(e.z), z1.y, acc);
+        acc = fmaf(ptx::bf16_lo(e.w), z1.z, acc);
+        acc = fmaf(ptx::bf16_hi(e.w), z1.w, acc);
+      }
       acc = warp_sum(acc);
       if (lane == 0) tgt_s[j][a] = acc - lse[static_cast<size_t>(i) * K + static_cast<size_t>(s) * r + a];
     }
