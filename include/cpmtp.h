@@ -41,7 +41,7 @@
  *    CPMTP_LSE_GROUP_MB, CPMTP_LSE_SPLITS and CPMTP_LSE_GROUP_TILES (schedule of the
  *    fused unembedding),
  *    CPMTP_GEMM_GROUP_ROWS (rows swept together by the other GEMMs), CPMTP_WIDE_MIN_K
- *    (shortest contraction that gets 256-row tiles), CPMTP_KL_GROUP_TILES and CPMTP_KL_SPLITS
+ *    and CPMTP_WIDE_MIN_ROWS (shortest contraction / fewest rows that get 256-row tiles), CPMTP_KL_GROUP_TILES and CPMTP_KL_SPLITS
  *    (schedule of the KL sweep of cpmtp_distill_forward; the latter also sizes its workspace).
  */
 #ifndef CPMTP_H

@@ -76,7 +76,12 @@ bool use_wide(long long rows, long long kdim) {
     const long long v = std::atoll(env);
     if (v >= 64) min_k = v;
   }
-  return rows >= 2 * kWideBM && kdim >= min_k;
+  long long min_rows = 2 * kWideBM;
+  if (const char* env = std::getenv("CPMTP_WIDE_MIN_ROWS")) {   // tuning knob
+    const long long v = std::atoll(env);
+    if (v > kBM) min_rows = v;
+  }
+  return rows >= min_rows && kdim >= min_k;
 }
 
 // Column-split schedule of the fused unembedding: `group` row tiles x `splits`
