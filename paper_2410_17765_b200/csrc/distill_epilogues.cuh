@@ -57,8 +57,8 @@ struct GroupLanes {
 };
 
 // l(v) = log p^d(v) - log p^c(v) for the W columns [col, col + W) this lane finishes; pd[i] holds
-// p^d on entry and l on exit.  Columns beyond V, rows beyond the last group and p^d = 0 (every
-// term underflowed; its weight in the sums is zero too) give l = 0.
+// p^d on entry and l on exit.  Columns beyond V, rows beyond the last group and a p^d below the
+// smallest normal float (every term underflowed; its weight in the sums is negligible too) give l = 0.
 // vec: V % 8 == 0, so the teacher row is 16-byte aligned and pieces of <= 8 columns never straddle V.
 template <int W>
 __device__ __forceinline__ void finish_columns(float* pd, const uint16_t* __restrict__ trow, int col, int V,
@@ -94,7 +94,7 @@ __device__ __forceinline__ void finish_columns(float* pd, const uint16_t* __rest
 #pragma unroll
     for (int i = 0; i < P; ++i) {
       const float p = pd[q * P + i];
-      const bool ok = row_ok && (c + i < V) && p > 0.f;
+      const bool ok = row_ok && (c + i < V) && p >= 1.17549435e-38f;   // lg2.approx flushes subnormals to -inf
       pd[q * P + i] = ok ? fmaf(ptx::lg2_approx(p), kLn2, lse_t - t[i]) : 0.f;
     }
   }

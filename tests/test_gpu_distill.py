@@ -140,3 +140,28 @@ def test_teacher_equal_to_own_conditional_gives_zero_kl():
     torch.cuda.synchronize()
     kl = out["kl"].cpu().numpy()
     assert np.max(np.abs(kl - ref.kl)) <= TOL and np.max(np.abs(kl)) < 5e-3
+
+
+def test_distill_stress_scale_stays_finite_and_tracks_the_bf16_z_oracle():
+    """Weights x 8: near one-hot factors, logits of several tens, mixture probabilities that underflow for
+    most of the vocabulary.  Everything must stay finite; the KL terms are compared with the oracle's bf16-z
+    mode (the exact mode differs by the rounding of z itself at this scale) relative to their size."""
+    from paper_2410_17765_b200 import binding
+
+    shape = synth.Shape(N=37, d=192, V=777, n=3, r=5)
+    inp = synth.make_inputs(shape, seed=2, weight_scale=8.0)
+    T = synth.make_teacher_logits(shape, inp.x, seed=2, std=6.0, target_bump=10.0)
+    dev = [t.cuda() for t in (inp.h, inp.W_head, inp.E, inp.W_g, inp.x, T)]
+    cs = binding.make_shape(shape.N, shape.d, shape.V, shape.n, shape.r)
+    saved, dsaved = binding.Saved.alloc(cs), binding.DistillSaved.alloc(cs)
+    st = torch.zeros(1, dtype=torch.int32, device="cuda")
+    out = binding.distill_forward(*dev, saved, dsaved, dev_status=st)
+    g = binding.distill_backward(*dev, saved, dsaved, dev_status=st)
+    torch.cuda.synchronize()
+    assert int(st.item()) == 0
+    kl = out["kl"].cpu().numpy()
+    assert np.all(np.isfinite(kl)) and np.isfinite(float(out["loss"].item()))
+    for key in ("dh", "dW_head", "dE", "dW_g"):
+        assert torch.isfinite(g[key].float()).all(), key
+    ref = distill.forward(inp.h, inp.W_head, inp.E, inp.W_g, inp.x, T, shape.n, shape.r, round_z=True)
+    assert np.max(np.abs(kl - ref.kl) / np.maximum(1.0, np.abs(ref.kl))) <= 5e-3
