@@ -64,32 +64,56 @@ def measured_peaks():
 
 
 class ClockSampler:
-    """nvidia-smi clock / throttle-reason samples taken while the timed region runs."""
+    """nvidia-smi clock / throttle-reason samples.  The query loop is started early (it needs a moment to come
+    up) and every sample is stamped on arrival; only those that arrived between begin() and end(), i.e. while
+    the timed region ran, are summarised."""
 
     FIELDS = ("clocks.sm,clocks.max.sm,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
               "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
 
     def __init__(self, gpu_index: int):
+        import threading
+
         self.proc = None
+        self.samples = []
+        self.t0 = self.t1 = None
         try:
             self.proc = subprocess.Popen(
                 ["nvidia-smi", f"--id={gpu_index}", f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits",
-                 "-lms", "50"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+                 "-lms", "20"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True, bufsize=1)
         except OSError:
             self.proc = None
+            return
+        self.thread = threading.Thread(target=self._read, daemon=True)
+        self.thread.start()
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.samples.append((time.perf_counter(), line))
+
+    def begin(self):
+        self.t0 = time.perf_counter()
+
+    def end(self):
+        self.t1 = time.perf_counter()
 
     def stop(self) -> dict:
         if self.proc is None:
             return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
         self.proc.terminate()
         try:
-            out, _ = self.proc.communicate(timeout=5)
+            self.proc.wait(timeout=5)
         except subprocess.TimeoutExpired:
             self.proc.kill()
-            out, _ = self.proc.communicate()
+        self.thread.join(timeout=5)
+        inside = [ln for t, ln in self.samples if self.t0 is not None and self.t0 <= t <= self.t1]
+        window = "timed region"
+        if not inside:   # region shorter than the query interval: the samples closest to it
+            inside = [ln for _, ln in self.samples[-3:]]
+            window = "last samples before the end of the timed region"
         sm, mx, reasons = [], [], set()
         names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
-        for line in out.strip().splitlines():
+        for line in inside:
             parts = [p.strip() for p in line.split(",")]
             if len(parts) < 6:
                 continue
@@ -102,7 +126,7 @@ class ClockSampler:
                 if val.lower().startswith("active"):
                     reasons.add(name)
         return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(mx) if mx else None,
-                "samples": len(sm), "reasons": sorted(reasons)}
+                "samples": len(sm), "window": window, "reasons": sorted(reasons)}
 
 
 def flops_per_position(s, kind, skip=()):
@@ -288,25 +312,29 @@ def run_ours(args, rank: int, world: int, local_rank: int):
         dist_util.barrier()
         torch.cuda.synchronize()
 
-    def timed(fn, steps, profile):
+    def timed(fn, steps, profile, clock_sampler=None):
         barrier()
         if profile:
             binding.profile_begin()
         e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        if clock_sampler is not None:
+            clock_sampler.begin()
         e0.record()
         for _ in range(steps):
             fn()
         e1.record()
         torch.cuda.synchronize()
+        if clock_sampler is not None:
+            clock_sampler.end()
         stages = binding.profile_end() if profile else {}
         ms = e0.elapsed_time(e1)
         barrier()
         return dist_util.max_over_ranks(ms, device), stages
 
+    sampler = ClockSampler(local_rank) if rank == 0 else None
     for _ in range(args.warmup):
         step()
-    sampler = ClockSampler(local_rank) if rank == 0 else None
-    ms_total, stages = timed(step, args.steps, True)
+    ms_total, stages = timed(step, args.steps, True, sampler)
     clocks = sampler.stop() if sampler is not None else None
     graph_ms = None
     if kind == "score" and not args.no_graph:   # launch-bound regime: the same step replayed from a CUDA graph
