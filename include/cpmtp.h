@@ -114,7 +114,7 @@ typedef struct cpmtp_saved {
 
 typedef struct CUstream_st* cpmtp_stream;
 
-int cpmtp_version(void);
+int cpmtp_version(void);   /* major * 100 + minor * 10; 110 added the distillation entry points */
 const char* cpmtp_status_string(int status);
 
 /* Scratch bytes needed by `op` (CPMTP_OP_*) for this shape; 0 if the shape is invalid. */

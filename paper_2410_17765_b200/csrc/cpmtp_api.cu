@@ -713,7 +713,7 @@ static int backward_impl(const cpmtp_shape* shape, const void* h, const void* W_
 
 extern "C" {
 
-int cpmtp_version(void) { return 100; }
+int cpmtp_version(void) { return 110; }   // 1.1: distillation entry points
 
 int cpmtp_profile_begin(void) {
   for (cudaEvent_t e : g_prof.events) cudaEventDestroy(e);
