@@ -131,19 +131,36 @@ __global__ void draft_step_partial_kernel(const float* __restrict__ S, int lds, 
   top.init();
   Cand best{-INFINITY, 0x7fffffff};
   const int v_end = min(V, (chunk + 1) * kSampleChunk);
-  for (int v = chunk * kSampleChunk + threadIdx.x; v < v_end; v += blockDim.x) {
-    float m = -INFINITY, l = 0.f;   // online logsumexp over the experts
+  // four consecutive vocabulary entries per thread and pass (lds % 32 == 0: 16-byte aligned loads; entries in
+  // [V, lds) exist in the buffer and are skipped below)
+  for (int v0 = chunk * kSampleChunk + 4 * threadIdx.x; v0 < v_end; v0 += 4 * blockDim.x) {
+    // two passes over the r logits (the second one hits L1): maximum first, then the sum of exponentials
+    float m[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
+#pragma unroll 4
     for (int a = 0; a < r; ++a) {
-      const float x = off_s[a] + Srow[static_cast<size_t>(a) * lds + v];
-      const float mn = fmaxf(m, x);
-      l = l * expf(m - mn) + expf(x - mn);
-      m = mn;
+      const float4 q = *reinterpret_cast<const float4*>(Srow + static_cast<size_t>(a) * lds + v0);
+      const float off = off_s[a];
+      m[0] = fmaxf(m[0], q.x + off); m[1] = fmaxf(m[1], q.y + off);
+      m[2] = fmaxf(m[2], q.z + off); m[3] = fmaxf(m[3], q.w + off);
     }
-    const float mix = m + logf(l);
-    top.insert(mix, v, topk);
-    float sc = mix;
-    if (urow != nullptr) sc = (mix - norm) * inv_temp - logf(-logf(urow[v]));
-    if (cand_better(sc, v, best.score, best.idx)) best = Cand{sc, v};
+    float l[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll 4
+    for (int a = 0; a < r; ++a) {
+      const float4 q = *reinterpret_cast<const float4*>(Srow + static_cast<size_t>(a) * lds + v0);
+      const float off = off_s[a];
+      l[0] += __expf(q.x + off - m[0]); l[1] += __expf(q.y + off - m[1]);
+      l[2] += __expf(q.z + off - m[2]); l[3] += __expf(q.w + off - m[3]);
+    }
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      const int v = v0 + j;
+      if (v >= v_end) continue;
+      const float mix = m[j] + __logf(l[j]);
+      top.insert(mix, v, topk);
+      float sc = mix;
+      if (urow != nullptr) sc = (mix - norm) * inv_temp - logf(-logf(urow[v]));
+      if (cand_better(sc, v, best.score, best.idx)) best = Cand{sc, v};
+    }
   }
   block_topk(top, topk, part_top + (static_cast<size_t>(i) * chunks + chunk) * kMaxTopk, red);
   const Cand b = block_best(best, red);
