@@ -337,7 +337,7 @@ def run_ours(args, rank: int, world: int, local_rank: int):
     ms_total, stages = timed(step, args.steps, True, sampler)
     clocks = sampler.stop() if sampler is not None else None
     graph_ms = None
-    if kind == "score" and not args.no_graph:   # launch-bound regime: the same step replayed from a CUDA graph
+    if kind in ("score", "sample") and not args.no_graph:   # launch-bound regime: the same step replayed from a CUDA graph
         side = torch.cuda.Stream()
         side.wait_stream(torch.cuda.current_stream())
         graph = torch.cuda.CUDAGraph()
