@@ -235,7 +235,7 @@ class Draft:
 
 
 def draft(h, W_head, E, W_g, n: int, r: int, *, topk: int = 1, uniform=None,
-          temperature: float = 1.0) -> Draft:
+          temperature: float = 1.0, forced=None) -> Draft:
     """Sequential draft generation from the factors (sampling section).
 
     The first token comes from the marginal of Eq. 11; for every later token the
@@ -250,6 +250,9 @@ def draft(h, W_head, E, W_g, n: int, r: int, *, topk: int = 1, uniform=None,
     distribution, sharpened by 1/temperature, with the Gumbel-max rule
     argmax_v( log p(v) / temperature - log(-log u[v]) ).
     topk: the k most likely tokens of each conditional (unperturbed), best first.
+    forced [N, n] int or None: entries >= 0 are taken as the drafted token of that step instead of the
+    selection (the candidates are still those of the conditional); -1 leaves the step to the sampler.  This is
+    how a caller walks a draft tree: the conditionals of a node are those given its path.
     """
     hd, Ed = _f64(h), _f64(E)
     N = hd.shape[0]
@@ -278,6 +281,9 @@ def draft(h, W_head, E, W_g, n: int, r: int, *, topk: int = 1, uniform=None,
             x_s = order[:, 0]
         else:
             x_s = np.argmax((mix - norm[:, None]) / temperature - np.log(-np.log(u[:, s, :])), axis=1)
+        if forced is not None:
+            f = _i64(forced)[:, s]
+            x_s = np.where(f >= 0, f, x_s)
         tokens[:, s] = x_s
         lb = lb + logP[rows, s, :, x_s]
     return Draft(tokens=tokens, logp_joint=logsumexp(lb, axis=1), topk_tokens=top_t, topk_logp=top_lp,

@@ -93,3 +93,33 @@ def test_gumbel_max_sampling_frequencies_match_the_joint():
     cold = cp_head.draft(inp.h, inp.W_head, inp.E, inp.W_g, s.n, s.r, uniform=u[:1], temperature=1e-6)
     greedy = cp_head.draft(inp.h, inp.W_head, inp.E, inp.W_g, s.n, s.r)
     assert np.array_equal(cold.tokens, greedy.tokens)
+
+
+def test_forced_prefix_gives_the_conditionals_of_that_path():
+    """With every token forced the joint score is the likelihood of that sequence (Eq. 9), and the candidates
+    of step s are the brute-force conditionals given the forced prefix; -1 entries fall back to the selection."""
+    import itertools
+
+    inp = synth.make_inputs(synth.Shape(3, 6, 5, 3, 3), seed=21, weight_scale=30.0)
+    s = inp.shape
+    args = (inp.h, inp.W_head, inp.E, inp.W_g)
+    rng = np.random.default_rng(3)
+    forced = rng.integers(0, s.V, size=(s.N, s.n))
+    out = cp_head.draft(*args, s.n, s.r, topk=s.V, forced=forced)
+    assert (out.tokens == forced).all()
+    fw = cp_head.forward(*args, forced.astype(np.int32), s.n, s.r)
+    assert np.allclose(out.logp_joint, fw.logp, atol=1e-12)
+    joint = np.empty((s.N,) + (s.V,) * s.n)
+    for tup in itertools.product(range(s.V), repeat=s.n):
+        xs = np.tile(np.array(tup, dtype=np.int32), (s.N, 1))
+        joint[(slice(None),) + tup] = np.exp(cp_head.forward(*args, xs, s.n, s.r).logp)
+    for i in range(s.N):
+        cond = joint[i, forced[i, 0], forced[i, 1]]
+        cond = cond / cond.sum()
+        order = out.topk_tokens[i, 2]
+        assert np.allclose(np.exp(out.topk_logp[i, 2]), cond[order], atol=1e-12)
+    partly = forced.copy()
+    partly[:, 1:] = -1
+    free = cp_head.draft(*args, s.n, s.r, topk=1, forced=partly)
+    assert (free.tokens[:, 0] == forced[:, 0]).all()
+    assert (free.tokens[:, 1] == out.topk_tokens[:, 1, 0]).all()   # greedy continuation of the forced first token
