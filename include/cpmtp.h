@@ -184,6 +184,10 @@ int cpmtp_score_draft(const cpmtp_shape* shape, const void* h, const void* W_hea
  *     Otherwise the token is argmax_v( log p(v) / temperature - log(-log uniform[v]) ),
  *     an exact draw from the conditional sharpened by 1/temperature (> 0).
  *   topk in [1, 8]: how many most-likely tokens of every conditional to report.
+ *   forced [N,n] int32 or NULL: an entry >= 0 is taken as the token of that step instead of the
+ *     selection (the candidates reported for the step are still those of the conditional); -1 leaves
+ *     the step to the sampler.  A caller walks a draft tree this way: the conditionals of a node are
+ *     those given its path.  Entries >= V are clamped to V-1 and raise dev_status 1.
  *   draft [N,n] int32 out.  logp_joint [N] fp32 out or NULL: Eq. 9 at the draft.
  *   topk_tokens [N,n,topk] int32 / topk_logp [N,n,topk] fp32 out or NULL: the
  *     candidates, best first, with their conditional log-probabilities (for a
@@ -191,7 +195,8 @@ int cpmtp_score_draft(const cpmtp_shape* shape, const void* h, const void* W_hea
  */
 int cpmtp_sample_draft(const cpmtp_shape* shape, const void* h, const void* W_head, const void* E,
                        const void* W_g, const float* uniform, float temperature, int32_t topk,
-                       int32_t* draft, float* logp_joint, int32_t* topk_tokens, float* topk_logp,
+                       const int32_t* forced, int32_t* draft, float* logp_joint, int32_t* topk_tokens,
+                       float* topk_logp,
                        void* workspace, size_t workspace_bytes, int32_t* dev_status,
                        cpmtp_stream stream);
 

@@ -80,8 +80,8 @@ def load_library() -> ctypes.CDLL:
     lib.cpmtp_forward_host.restype = ctypes.c_int
     lib.cpmtp_forward_host.argtypes = [shp, vp, vp, vp, vp, i32p, fp, fp, svp, vp, sz, i32p, vp]
     lib.cpmtp_sample_draft.restype = ctypes.c_int
-    lib.cpmtp_sample_draft.argtypes = [shp, vp, vp, vp, vp, fp, ctypes.c_float, ctypes.c_int32, i32p, fp, i32p, fp,
-                                       vp, sz, i32p, vp]
+    lib.cpmtp_sample_draft.argtypes = [shp, vp, vp, vp, vp, fp, ctypes.c_float, ctypes.c_int32, i32p, i32p, fp, i32p,
+                                       fp, vp, sz, i32p, vp]
     lib.cpmtp_forward_full.restype = ctypes.c_int
     lib.cpmtp_forward_full.argtypes = [shp, vp, vp, vp, i32p, fp, fp, fp, svp, i32p, vp, sz, i32p, vp]
     lib.cpmtp_backward_full.restype = ctypes.c_int
@@ -280,10 +280,11 @@ def score_draft(h, W_head, E, W_g, draft, *, want_prefix: bool = True,
 
 
 def sample_draft(h, W_head, E, W_g, n: int, *, uniform: Optional[torch.Tensor] = None, temperature: float = 1.0,
-                 topk: int = 1, workspace: Optional[torch.Tensor] = None,
+                 topk: int = 1, forced: Optional[torch.Tensor] = None, workspace: Optional[torch.Tensor] = None,
                  dev_status: Optional[torch.Tensor] = None, out: Optional[dict] = None) -> dict:
     """cpmtp_sample_draft; returns {"draft", "logp_joint", "topk_tokens", "topk_logp"} (device tensors).
-    uniform: [N, n, V] fp32 strictly inside (0, 1) for Gumbel-max sampling, or None for the greedy draft."""
+    uniform: [N, n, V] fp32 strictly inside (0, 1) for Gumbel-max sampling, or None for the greedy draft.
+    forced: [N, n] int32, entries >= 0 fix the token of that step (-1: left to the sampler), or None."""
     lib = load_library()
     N, d = h.shape
     V, r = E.shape[0], W_g.shape[0]
@@ -292,6 +293,8 @@ def sample_draft(h, W_head, E, W_g, n: int, *, uniform: Optional[torch.Tensor] =
         assert t.dtype == torch.bfloat16 and t.is_contiguous()
     if uniform is not None:
         assert uniform.shape == (N, n, V) and uniform.dtype == torch.float32 and uniform.is_contiguous()
+    if forced is not None:
+        assert forced.shape == (N, n) and forced.dtype == torch.int32 and forced.is_contiguous()
     shape = make_shape(N, d, V, n, r)
     if workspace is None:
         workspace = alloc_workspace(workspace_bytes(shape, OP_SAMPLE), h.device)
@@ -302,7 +305,8 @@ def sample_draft(h, W_head, E, W_g, n: int, *, uniform: Optional[torch.Tensor] =
     res.setdefault("topk_tokens", torch.empty((N, n, topk), dtype=torch.int32, device=dev))
     res.setdefault("topk_logp", torch.empty((N, n, topk), dtype=torch.float32, device=dev))
     rc = lib.cpmtp_sample_draft(ctypes.byref(shape), _ptr(h), _ptr(W_head), _ptr(E), _ptr(W_g), _ptr(uniform),
-                                ctypes.c_float(temperature), topk, _ptr(res["draft"]), _ptr(res["logp_joint"]),
+                                ctypes.c_float(temperature), topk, _ptr(forced), _ptr(res["draft"]),
+                                _ptr(res["logp_joint"]),
                                 _ptr(res["topk_tokens"]), _ptr(res["topk_logp"]), _ptr(workspace), workspace.numel(),
                                 _ptr(dev_status), _stream())
     _check(rc)

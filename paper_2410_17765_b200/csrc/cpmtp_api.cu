@@ -819,8 +819,9 @@ int cpmtp_score_draft(const cpmtp_shape* shape, const void* h, const void* W_hea
 }
 
 int cpmtp_sample_draft(const cpmtp_shape* shape, const void* h, const void* W_head, const void* E,
-                       const void* W_g, const float* uniform, float temperature, int32_t topk, int32_t* draft,
-                       float* logp_joint, int32_t* topk_tokens, float* topk_logp, void* workspace,
+                       const void* W_g, const float* uniform, float temperature, int32_t topk,
+                       const int32_t* forced, int32_t* draft, float* logp_joint, int32_t* topk_tokens,
+                       float* topk_logp, void* workspace,
                        size_t workspace_bytes, int32_t* dev_status, cpmtp_stream stream) {
   DeviceInfo* di = nullptr;
   const int rc = check_common(shape, h, W_head, E, W_g, /*x=*/h, workspace, &di);
@@ -856,7 +857,8 @@ int cpmtp_sample_draft(const cpmtp_shape* shape, const void* h, const void* W_he
     draft_step_final_kernel<<<s.N, kSampleFinalThreads, 0, st>>>(z32, static_cast<const uint16_t*>(E), s.d, lse, lb,
                                                            part_top, part_best, L.chunks,
                                                            uniform != nullptr ? 1 : 0, step, s.V, s.n, s.r, topk,
-                                                           draft, logp_joint, topk_tokens, topk_logp);
+                                                           forced, dev_status, draft, logp_joint, topk_tokens,
+                                                           topk_logp);
     CPMTP_TRY(cudaGetLastError());
   }
   return CPMTP_OK;

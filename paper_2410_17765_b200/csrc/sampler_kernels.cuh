@@ -176,7 +176,8 @@ __global__ void __launch_bounds__(kSampleFinalThreads) draft_step_final_kernel(c
                                         const float* __restrict__ lse,
                                         float* __restrict__ lb, const Cand* __restrict__ part_top,
                                         const Cand* __restrict__ part_best, int chunks, int sampled, int s, int V,
-                                        int n, int r, int topk, int32_t* __restrict__ draft,
+                                        int n, int r, int topk, const int32_t* __restrict__ forced,
+                                        int* __restrict__ dev_status, int32_t* __restrict__ draft,
                                         float* __restrict__ logp_joint, int32_t* __restrict__ topk_tokens,
                                         float* __restrict__ topk_logp) {
   __shared__ Cand red[32];
@@ -206,7 +207,19 @@ __global__ void __launch_bounds__(kSampleFinalThreads) draft_step_final_kernel(c
     const float tot = warp_sum(e);
     if (a == 0) norm_s = m + logf(tot);
   }
-  if (threadIdx.x == 0) cand_tok[topk] = sampled ? b.idx : final_top[0].idx;   // the drafted token
+  if (threadIdx.x == 0) {   // the drafted token: the caller's, if one is given for this step
+    int tok = sampled ? b.idx : final_top[0].idx;
+    if (forced != nullptr) {
+      const int f = forced[static_cast<size_t>(i) * n + s];
+      if (f >= V) {
+        if (dev_status != nullptr) atomicMax(dev_status, 1);   // out of range: clamped and reported
+        tok = V - 1;
+      } else if (f >= 0) {
+        tok = f;
+      }
+    }
+    cand_tok[topk] = tok;
+  }
   if (threadIdx.x < topk) cand_tok[threadIdx.x] = final_top[threadIdx.x].idx;
   __syncthreads();
   // Exact logits (from the unrounded z) of the candidates and of the drafted token, for every expert.

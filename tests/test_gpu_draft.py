@@ -131,3 +131,34 @@ def test_verify_draft_matches_oracle():
     assert clear.mean() > 0.99
     assert np.array_equal(got[clear], want[clear])
     assert got.min() >= 0 and got.max() <= n
+
+
+def test_forced_tokens_walk_a_draft_tree():
+    """Forced entries replace the selection; the reported candidates are the conditionals given the forced path
+    and the joint score is the likelihood of the path; -1 entries are left to the sampler."""
+    from paper_2410_17765_b200 import binding
+
+    shape = synth.Shape(N=6, d=256, V=1500, n=3, r=4)
+    inp = synth.make_inputs(shape, seed=11, weight_scale=2.0)
+    dev = to_dev(inp)
+    g = torch.Generator().manual_seed(5)
+    forced = torch.randint(0, shape.V, (shape.N, shape.n), generator=g, dtype=torch.int32)
+    forced[::2, 1:] = -1                     # every other position: only the first token is given
+    ref = cp_head.draft(inp.h, inp.W_head, inp.E, inp.W_g, shape.n, shape.r, topk=4, forced=forced)
+    st = torch.zeros(1, dtype=torch.int32, device="cuda")
+    out = binding.sample_draft(*dev, shape.n, topk=4, forced=forced.cuda(), dev_status=st)
+    torch.cuda.synchronize()
+    assert int(st.item()) == 0
+    draft = out["draft"].cpu()
+    given = forced >= 0
+    assert torch.equal(draft[given], forced[given])
+    assert np.array_equal(draft.numpy(), ref.tokens)
+    assert np.max(np.abs(out["logp_joint"].cpu().numpy() - ref.logp_joint)) <= 2e-3
+    assert np.array_equal(out["topk_tokens"].cpu().numpy(), ref.topk_tokens)
+    assert np.max(np.abs(out["topk_logp"].cpu().numpy() - ref.topk_logp)) <= 2e-3
+    # a token beyond the vocabulary is clamped and reported
+    bad = forced.clone()
+    bad[0, 0] = shape.V + 7
+    out2 = binding.sample_draft(*dev, shape.n, topk=1, forced=bad.cuda(), dev_status=st)
+    torch.cuda.synchronize()
+    assert int(st.item()) == 1 and int(out2["draft"][0, 0].item()) == shape.V - 1
