@@ -91,3 +91,27 @@ def test_distill_workspace_and_argument_checks(lib):
                                      p, 4096, None, None) in (-1, -5, -6)
     assert lib.cpmtp_distill_backward(ctypes.byref(s), p, p, p, p, p, None, None, None, f(0.9), f(1.0), None, None,
                                       p, p, p, p, p, 4096, None, None) == -1
+
+
+def test_product_and_oracle_do_not_import_each_other():
+    """The package never imports the oracle (no CPU fallback can hide behind it) and the oracle never imports the
+    package's CUDA side; only the seeded input generators are shared."""
+    import ast
+    import pathlib
+
+    root = pathlib.Path(__file__).resolve().parents[1]
+
+    def imported(path):
+        names = set()
+        for node in ast.walk(ast.parse(path.read_text())):
+            if isinstance(node, ast.Import):
+                names.update(a.name for a in node.names)
+            elif isinstance(node, ast.ImportFrom):
+                names.add(("." * node.level) + (node.module or ""))
+                names.update(f"{node.module or ''}.{a.name}" for a in node.names)
+        return names
+
+    for f in (root / "paper_2410_17765_b200").glob("*.py"):
+        assert not any(n.split(".")[0] == "oracle" or ".oracle" in n for n in imported(f)), f
+    for f in (root / "oracle").glob("*.py"):
+        assert not any("binding" in n or "build" in n or "dist_util" in n for n in imported(f)), f
