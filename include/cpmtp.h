@@ -32,9 +32,12 @@
  *    capture and replayed (same pointers, new contents); call each once outside capture first, since the
  *    first launch of a kernel sets its shared-memory attribute.  Environment knobs are read at capture time.
  *  - Threads: calls may be made from several host threads as long as each uses
- *    its own stream, workspace and outputs; the per-stage profiling calls are
- *    the exception (one thread, one device).
- *  - Environment knobs, read at call time, for testing and tuning only:
+ *    its own stream, workspace and outputs (the library's few host-side caches --
+ *    device properties, kernel attributes, tensor maps -- are guarded by a lock); the
+ *    per-stage profiling calls and cpmtp_reload_knobs are the exception (one thread,
+ *    no other call in flight).
+ *  - Environment knobs, for testing and tuning only.  They are read ONCE, at the first call
+ *    into the library; cpmtp_reload_knobs() reads them again.
  *    CPMTP_BWD_CHUNK_ROWS / CPMTP_BWD_CHUNK_HEADS (rows / heads of logit gradients
  *    recomputed at a time in the backward passes; also changes the workspace the
  *    backward needs, so set it before querying cpmtp_workspace_bytes),
@@ -42,7 +45,17 @@
  *    fused unembedding),
  *    CPMTP_GEMM_GROUP_ROWS (rows swept together by the other GEMMs), CPMTP_WIDE_MIN_K
  *    and CPMTP_WIDE_MIN_ROWS (shortest contraction / fewest rows that get 256-row tiles), CPMTP_KL_GROUP_TILES and CPMTP_KL_SPLITS
- *    (schedule of the KL sweep of cpmtp_distill_forward; the latter also sizes its workspace).
+ *    (schedule of the KL sweep of cpmtp_distill_forward; the latter also sizes its workspace),
+ *    CPMTP_WAIT_LIMIT_US (how long a wait inside a kernel may last before the kernel gives up with
+ *    device status 2; default 4 s) and CPMTP_TEST_SKIP_LOAD (test hook: every CTA of the tensor-core
+ *    kernels leaves out that one operand load, so the give-up path runs; results are invalid).
+ *  - Accuracy: log-probabilities are within 2e-3 of the exact definition and gradients within 1e-2
+ *    relative L2 at the weight scales of trained heads (logit standard deviation of a few units) when
+ *    V is in the thousands or more.  The projected hidden state z is held in bf16 between the two
+ *    products; a vocabulary-wide logsumexp averages that rounding out, but with d >= 4096 and only a few
+ *    hundred vocabulary entries it does not: there logsumexp_v can be off by up to 2e-3 and the KL terms
+ *    of cpmtp_distill_forward by up to 2e-2.  The target logits are taken from the unrounded z and the
+ *    full-head entry points have no bf16 intermediate.
  */
 #ifndef CPMTP_H
 #define CPMTP_H
@@ -90,6 +103,12 @@ enum {
  * N*n*r*d*2 bytes while the saved state shrinks by as much; +2*N*n*r*d*d flop).  Set the flag in
  * both calls and in the workspace query. */
 #define CPMTP_FLAG_RECOMPUTE_Z 4u
+/* Backward entry points: add the gradients to what dh / dW_head (dW_full) / dE / dW_g already hold instead
+ * of overwriting them (gradient accumulation over micro-batches, the usual way the training objective of
+ * Eq. 9 is run at more positions than one call holds).  The sum is formed in fp32 from the stored bf16
+ * value and this call's fp32 accumulator and rounded to bf16 once per call; the caller zeroes the buffers
+ * before the first micro-batch. */
+#define CPMTP_FLAG_ACCUM_GRADS 8u
 
 typedef struct cpmtp_shape {
   int32_t N;        /* positions */
@@ -114,8 +133,13 @@ typedef struct cpmtp_saved {
 
 typedef struct CUstream_st* cpmtp_stream;
 
-int cpmtp_version(void);   /* major * 100 + minor * 10; 110 added the distillation entry points */
+int cpmtp_version(void);   /* major * 100 + minor * 10; 110 added the distillation entry points, 120 CPMTP_FLAG_ACCUM_GRADS */
 const char* cpmtp_status_string(int status);
+
+/* Read the environment knobs listed above again (they are otherwise read once per process).  For tests
+ * and tuning runs that change a knob between calls; not to be called while another call is in flight.
+ * The paper has no counterpart for this call. */
+int cpmtp_reload_knobs(void);
 
 /* Scratch bytes needed by `op` (CPMTP_OP_*) for this shape; 0 if the shape is invalid. */
 size_t cpmtp_workspace_bytes(const cpmtp_shape* shape, int op);
@@ -178,7 +202,7 @@ int cpmtp_score_draft(const cpmtp_shape* shape, const void* h, const void* W_hea
  * drawn, as the text under Eq. 12 describes (the printed Eq. 12 / Eq. 13 lack the
  * s-th factor and the normaliser).  E and W_head are streamed once; the logits of
  * the N*n*r rows are kept in the workspace (fp32) for the n sequential steps, so
- * this entry point is meant for decode-sized N.
+ * this entry point is meant for decode-sized N (N <= 65535, else CPMTP_ERR_LIMIT).
  *   uniform [N,n,V] fp32, every value strictly inside (0,1), or NULL.  NULL: the
  *     most likely token is taken (temperature 0; ties go to the lowest id).
  *     Otherwise the token is argmax_v( log p(v) / temperature - log(-log uniform[v]) ),
@@ -243,7 +267,8 @@ int cpmtp_backward_full(const cpmtp_shape* shape, const void* h, const void* W_f
  *   saved and dsaved are required and are filled for cpmtp_distill_backward.
  * The vocabulary is swept twice: the fused log-sum-exp pass of cpmtp_forward, then a pass in which
  * the r experts of a (position, token) pair occupy adjacent accumulator rows (padded to a power of
- * two) and are mixed across lanes, so p^d and the logits are never written to memory either.
+ * two) and are mixed across lanes, so p^d and the logits are never written to memory either.  The teacher
+ * logits are read once, in that second pass, which also accumulates their logsumexp (dsaved->lse_t).
  * Workspace: CPMTP_OP_DISTILL_FORWARD.  CPMTP_FLAG_RECOMPUTE_Z is honoured as in cpmtp_forward.
  */
 typedef struct cpmtp_distill_saved {
@@ -307,8 +332,10 @@ int cpmtp_verify_draft(int32_t N, int32_t n, const int32_t* draft, const int32_t
  *    nothing is enqueued.  At d = 4096, n*r = 32 that allows up to 8 positions.
  *  - No cudaMalloc / cudaFree or other allocating call is made, on any call.
  *  - The first call on each device looks up the array's device address (a
- *    one-time host-side query, made with that device current).  Make that first
- *    call outside any stream capture.
+ *    one-time host-side query, made with that device current, guarded by the
+ *    library's cache lock).  Make that first call outside any stream capture.
+ *    The address is kept for the life of the process: do not call
+ *    cudaDeviceReset() between calls.
  *  - All calls on a device share the one array, which keeps whatever the
  *    previous call left in it.  Every location is written before it is read
  *    within a call, so nothing needs clearing; but two calls that overlap on the
@@ -361,7 +388,7 @@ enum {
   CPMTP_STAGE_DH,
   CPMTP_STAGE_DW_G,
   CPMTP_STAGE_DRAFT_STEP,    /* per-token selection passes of cpmtp_sample_draft */
-  CPMTP_STAGE_TEACHER_LSE,   /* logsumexp_V of the teacher logits + expert weights per token (Eq. 14) */
+  CPMTP_STAGE_TEACHER_LSE,   /* expert weights per token (Eq. 14); the teacher's logsumexp_V is part of the KL pass */
   CPMTP_STAGE_KL,            /* second unembedding pass: KL term of Eq. 14 */
   CPMTP_STAGE_COUNT
 };

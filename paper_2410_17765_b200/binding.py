@@ -6,6 +6,7 @@ library is missing or fails to load, importing this module's functions raises.
 """
 from __future__ import annotations
 
+import contextlib
 import ctypes
 import os
 from dataclasses import dataclass
@@ -20,13 +21,14 @@ OP_DISTILL_FORWARD, OP_DISTILL_BACKWARD = 6, 7
 FLAG_AUX = 1
 FLAG_PER_TOKEN = 2
 FLAG_RECOMPUTE_Z = 4
+FLAG_ACCUM_GRADS = 8
 
 EXPORTS = [
     "cpmtp_version", "cpmtp_status_string", "cpmtp_workspace_bytes", "cpmtp_forward", "cpmtp_backward",
     "cpmtp_score_draft", "cpmtp_host_staging_bytes", "cpmtp_forward_host", "cpmtp_profile_begin",
     "cpmtp_profile_end", "cpmtp_score_draft_static", "cpmtp_sample_draft",
     "cpmtp_forward_full", "cpmtp_backward_full", "cpmtp_verify_draft",
-    "cpmtp_distill_forward", "cpmtp_distill_backward",
+    "cpmtp_distill_forward", "cpmtp_distill_backward", "cpmtp_reload_knobs",
 ]
 
 STATIC_SCRATCH_BYTES = 4 << 20
@@ -97,11 +99,37 @@ def load_library() -> ctypes.CDLL:
     lib.cpmtp_distill_backward.restype = ctypes.c_int
     lib.cpmtp_distill_backward.argtypes = [shp, vp, vp, vp, vp, i32p, vp, svp, dsp, ctypes.c_float, ctypes.c_float,
                                            fp, fp, vp, vp, vp, vp, vp, sz, i32p, vp]
+    lib.cpmtp_reload_knobs.restype = ctypes.c_int
     lib.cpmtp_profile_begin.restype = ctypes.c_int
     lib.cpmtp_profile_end.restype = ctypes.c_int
     lib.cpmtp_profile_end.argtypes = [ctypes.POINTER(ctypes.c_float), ctypes.POINTER(ctypes.c_int32), ctypes.c_int]
     _lib = lib
     return lib
+
+
+def reload_knobs() -> None:
+    """cpmtp_reload_knobs: have the library read its CPMTP_* environment knobs again."""
+    _check(load_library().cpmtp_reload_knobs())
+
+
+@contextlib.contextmanager
+def knobs(**values):
+    """Set CPMTP_* environment knobs (name=value; None leaves a knob alone) for the calls made inside the
+    block, then restore the environment; the library re-reads its knobs on entry and on exit."""
+    values = {k: v for k, v in values.items() if v is not None}
+    old = {k: os.environ.get(k) for k in values}
+    try:
+        for k, v in values.items():
+            os.environ[k] = str(v)
+        reload_knobs()
+        yield
+    finally:
+        for k, v in old.items():
+            if v is None:
+                os.environ.pop(k, None)
+            else:
+                os.environ[k] = v
+        reload_knobs()
 
 
 def profile_begin() -> None:
@@ -232,14 +260,18 @@ def backward(h, W_head, E, W_g, x, saved: Saved, *, aux_coef: Optional[float] = 
              dloss_dlogp: Optional[torch.Tensor] = None, workspace: Optional[torch.Tensor] = None,
              dev_status: Optional[torch.Tensor] = None, out: Optional[dict] = None,
              skip: tuple = (), dloss_dprefix: Optional[torch.Tensor] = None,
-             recompute_z: bool = False) -> dict:
+             recompute_z: bool = False, accumulate: bool = False) -> dict:
     """cpmtp_backward on device tensors; returns {"dh", "dW_head", "dE", "dW_g"} (bf16 device tensors).
     Names listed in `skip` are not computed (passed as NULL).  dloss_dprefix [N, n] fp32 selects the
-    per-token objective sum_i sum_s dloss_dprefix[i, s] * log P(x[i, 0..s]) (CPMTP_FLAG_PER_TOKEN)."""
+    per-token objective sum_i sum_s dloss_dprefix[i, s] * log P(x[i, 0..s]) (CPMTP_FLAG_PER_TOKEN).
+    accumulate: add to the tensors given in `out` instead of overwriting them (CPMTP_FLAG_ACCUM_GRADS)."""
     lib = load_library()
     shape = _shape_of(h, W_head, E, W_g, x, aux_coef)
     if recompute_z:
         shape.flags |= FLAG_RECOMPUTE_Z
+    if accumulate:
+        assert out is not None, "accumulation needs the tensors to add to"
+        shape.flags |= FLAG_ACCUM_GRADS
     if dloss_dprefix is not None:
         assert dloss_dlogp is None and dloss_dprefix.shape == (shape.N, shape.n) and dloss_dprefix.dtype == torch.float32
         shape.flags |= FLAG_PER_TOKEN
@@ -351,11 +383,14 @@ def forward_full(h, W_full, W_g, x, *, aux_coef: Optional[float] = None, saved: 
 def backward_full(h, W_full, W_g, x, saved: Saved, *, aux_coef: Optional[float] = None,
                   dloss_dlogp: Optional[torch.Tensor] = None, workspace: Optional[torch.Tensor] = None,
                   dev_status: Optional[torch.Tensor] = None, out: Optional[dict] = None,
-                  dloss_dprefix: Optional[torch.Tensor] = None) -> dict:
+                  dloss_dprefix: Optional[torch.Tensor] = None, accumulate: bool = False) -> dict:
     """cpmtp_backward_full; returns {"dh", "dW_full", "dW_g"} (bf16 device tensors).
-    dloss_dprefix as for backward()."""
+    dloss_dprefix and accumulate as for backward()."""
     lib = load_library()
     shape = _shape_full(h, W_full, W_g, x, aux_coef)
+    if accumulate:
+        assert out is not None, "accumulation needs the tensors to add to"
+        shape.flags |= FLAG_ACCUM_GRADS
     if dloss_dprefix is not None:
         assert dloss_dlogp is None and dloss_dprefix.shape == (shape.N, shape.n) and dloss_dprefix.dtype == torch.float32
         shape.flags |= FLAG_PER_TOKEN
@@ -487,13 +522,17 @@ def distill_backward(h, W_head, E, W_g, x, teacher, saved: Saved, dsaved: Distil
                      gamma: float = 1.0, aux_coef: Optional[float] = None,
                      dloss_dprefix: Optional[torch.Tensor] = None, dloss_dkl: Optional[torch.Tensor] = None,
                      workspace: Optional[torch.Tensor] = None, dev_status: Optional[torch.Tensor] = None,
-                     out: Optional[dict] = None, skip: tuple = (), recompute_z: bool = False) -> dict:
+                     out: Optional[dict] = None, skip: tuple = (), recompute_z: bool = False,
+                     accumulate: bool = False) -> dict:
     """cpmtp_distill_backward; returns {"dh", "dW_head", "dE", "dW_g"} (bf16 device tensors)."""
     lib = load_library()
     shape = _shape_of(h, W_head, E, W_g, x, aux_coef)
     _check_teacher(teacher, shape)
     if recompute_z:
         shape.flags |= FLAG_RECOMPUTE_Z
+    if accumulate:
+        assert out is not None, "accumulation needs the tensors to add to"
+        shape.flags |= FLAG_ACCUM_GRADS
     for w in (dloss_dprefix, dloss_dkl):
         assert w is None or (w.shape == (shape.N, shape.n) and w.dtype == torch.float32 and w.is_contiguous())
     if workspace is None:

@@ -6,6 +6,8 @@
 #include <cuda_runtime.h>
 #include <cstdint>
 #include <cstdlib>
+#include <cstring>
+#include <mutex>
 #include <vector>
 
 #include "distill_epilogues.cuh"
@@ -22,15 +24,16 @@ namespace {
 constexpr int kBN = 256;
 constexpr int kStages = 4;
 constexpr size_t kAlign = 256;
-constexpr size_t kLogitGradBudgetBytes = 4ull << 30;   // bound on the recomputed-logit-gradient chunk
+// Bound on the chunk of recomputed logit gradients (bf16) that the backward holds at a time.  Large on
+// purpose (the device has 180 GB): every chunk costs one read-modify-write of the fp32 dE accumulator and a
+// partly filled last wave in each of its GEMMs, so few, long chunks are cheaper than many short ones.
+constexpr size_t kLogitGradBudgetBytes = 16ull << 30;
 
 using CfgKK = TileCfg<kBN, kStages, false, false>;   // A K-major, B K-major
 constexpr int kWideStages = 3;                        // 64 KB per slot
 constexpr int kWideBM = 2 * kBM;
-using WideKK = TileCfg<kBN, kWideStages, false, false, kBM, 2>;   // 256 x 256 tiles, two row blocks share B
 using CfgKKSkinny = TileCfg<kBN, 5, false, false, 32>;   // <= 32 rows of A: bandwidth-bound draft scoring
-using CfgKM = TileCfg<kBN, kStages, false, true>;    // A K-major, B MN-major
-using CfgMM = TileCfg<kBN, kStages, true, true>;     // both MN-major
+using WideKK = TileCfg<kBN, kWideStages, false, false, kBM, 2>;   // 256 x 256 tiles, two row blocks share B
 
 inline size_t align_up(size_t v, size_t a = kAlign) { return (v + a - 1) / a * a; }
 
@@ -40,11 +43,16 @@ struct DeviceInfo {
   bool ok = false;
 };
 
+// One lock for the small per-process caches below (device properties, kernel attributes, tensor maps,
+// the static scratch address).  Host-side only and held for microseconds; calls from several threads are safe.
+std::mutex g_cache_mutex;
+
 // Cached per device ordinal; filled on first use with that device current.
 DeviceInfo* device_info() {
   static DeviceInfo infos[64];
   int dev = 0;
   if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return nullptr;
+  std::lock_guard<std::mutex> lock(g_cache_mutex);
   DeviceInfo& di = infos[dev];
   if (!di.ok) {
     if (cudaDeviceGetAttribute(&di.sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return nullptr;
@@ -53,6 +61,51 @@ DeviceInfo* device_info() {
     di.ok = true;
   }
   return &di;
+}
+
+// Testing / tuning knobs from the environment, read once per process (and again by cpmtp_reload_knobs);
+// 0 = not set.
+struct Knobs {
+  long long wide_min_k = 0, wide_min_rows = 0;
+  long long lse_group_mb = 0, lse_splits = 0, lse_group_tiles = 0;
+  long long bwd_chunk_rows = 0, bwd_chunk_heads = 0, gemm_group_rows = 0;
+  long long kl_group_tiles = 0, kl_splits = 0;
+  long long wait_limit_us = 0, test_skip_load = 0;
+  long long proj_tiles = 0;
+};
+Knobs g_knobs;
+std::once_flag g_knobs_once;
+
+void read_knobs() {
+  auto get = [](const char* name) -> long long {
+    const char* v = std::getenv(name);
+    return v != nullptr ? std::atoll(v) : 0;
+  };
+  Knobs k;
+  k.wide_min_k = get("CPMTP_WIDE_MIN_K");
+  k.wide_min_rows = get("CPMTP_WIDE_MIN_ROWS");
+  k.lse_group_mb = get("CPMTP_LSE_GROUP_MB");
+  k.lse_splits = get("CPMTP_LSE_SPLITS");
+  k.lse_group_tiles = get("CPMTP_LSE_GROUP_TILES");
+  k.bwd_chunk_rows = get("CPMTP_BWD_CHUNK_ROWS");
+  k.bwd_chunk_heads = get("CPMTP_BWD_CHUNK_HEADS");
+  k.gemm_group_rows = get("CPMTP_GEMM_GROUP_ROWS");
+  k.kl_group_tiles = get("CPMTP_KL_GROUP_TILES");
+  k.kl_splits = get("CPMTP_KL_SPLITS");
+  k.wait_limit_us = get("CPMTP_WAIT_LIMIT_US");
+  k.test_skip_load = get("CPMTP_TEST_SKIP_LOAD");
+  k.proj_tiles = get("CPMTP_PROJ_TILE_ROWS");
+  g_knobs = k;
+}
+
+const Knobs& knobs() {
+  std::call_once(g_knobs_once, read_knobs);
+  return g_knobs;
+}
+
+int sms_or_default() {
+  DeviceInfo* di = device_info();
+  return (di != nullptr && di->sms > 0) ? di->sms : 148;
 }
 
 int validate_shape(const cpmtp_shape* s) {
@@ -72,15 +125,9 @@ inline bool aligned(const void* p, size_t a) { return (reinterpret_cast<uintptr_
 // amortise it; otherwise 128-row tiles with the double-buffered accumulator are used.
 bool use_wide(long long rows, long long kdim) {
   long long min_k = 4096;
-  if (const char* env = std::getenv("CPMTP_WIDE_MIN_K")) {   // tuning knob
-    const long long v = std::atoll(env);
-    if (v >= 64) min_k = v;
-  }
+  if (knobs().wide_min_k >= 64) min_k = knobs().wide_min_k;   // tuning knob
   long long min_rows = 2 * kWideBM;
-  if (const char* env = std::getenv("CPMTP_WIDE_MIN_ROWS")) {   // tuning knob
-    const long long v = std::atoll(env);
-    if (v > kBM) min_rows = v;
-  }
+  if (knobs().wide_min_rows > kBM) min_rows = knobs().wide_min_rows;   // tuning knob
   return rows >= min_rows && kdim >= min_k;
 }
 
@@ -98,10 +145,7 @@ Sched sched_lse(int m_tiles, int n_tiles, int M, int V, int d, int bm, int slots
   // least DRAM traffic and the best time at V = 32000 and V = 128256; larger groups start to
   // evict one another's z tiles and the E stream.  The 0.5 MB tiles at d = 2048 did best with 64 MB.
   long long l2_budget_mb = bm > kBM ? 24 : 64;
-  if (const char* env = std::getenv("CPMTP_LSE_GROUP_MB")) {   // tuning knob: L2 budget for the swept z tiles
-    const long long v = std::atoll(env);
-    if (v >= 1 && v <= 1024) l2_budget_mb = v;
-  }
+  if (knobs().lse_group_mb >= 1 && knobs().lse_group_mb <= 1024) l2_budget_mb = knobs().lse_group_mb;   // tuning knob
   int max_group = static_cast<int>((l2_budget_mb << 20) / (2ll * bm * d));
   if (max_group < 1) max_group = 1;
   const double tile_t = 2.0 * bm * kBN * d / (1.4e15 / 148.0);
@@ -123,10 +167,7 @@ Sched sched_lse(int m_tiles, int n_tiles, int M, int V, int d, int bm, int slots
       best_ctas = ctas;
     }
   }
-  if (const char* env = std::getenv("CPMTP_LSE_SPLITS")) {   // tuning knob: force the split count
-    const int v = std::atoi(env);
-    if (v >= 1 && v <= s_max) best_s = v;
-  }
+  if (knobs().lse_splits >= 1 && knobs().lse_splits <= s_max) best_s = static_cast<int>(knobs().lse_splits);   // tuning knob
   int group = static_cast<long long>(m_tiles) * best_s >= sms ? (sms / best_s) : m_tiles;
   if (bm > kBM && m_tiles >= 8) {
     // 256-row tiles (d >= 4096): measured on B200, short units in the raster of the plain GEMMs beat
@@ -136,15 +177,9 @@ Sched sched_lse(int m_tiles, int n_tiles, int M, int V, int d, int bm, int slots
     group = 8;
     best_s = n_tiles < 125 ? n_tiles : 125;
     if ((static_cast<long long>(group) * best_s) % sms == 0 && best_s > 1) --best_s;
-    if (const char* env2 = std::getenv("CPMTP_LSE_SPLITS")) {
-      const int v = std::atoi(env2);
-      if (v >= 1 && v <= n_tiles) best_s = v;
-    }
+    if (knobs().lse_splits >= 1 && knobs().lse_splits <= n_tiles) best_s = static_cast<int>(knobs().lse_splits);
   }
-  if (const char* env = std::getenv("CPMTP_LSE_GROUP_TILES")) {   // tuning knob: force the row group
-    const int v = std::atoi(env);
-    if (v >= 1) group = v;
-  }
+  if (knobs().lse_group_tiles >= 1) group = static_cast<int>(knobs().lse_group_tiles);   // tuning knob: force the row group
   return make_sched(m_tiles, n_tiles, best_s, group < 1 ? 1 : group, d / kBK);
 }
 
@@ -153,6 +188,7 @@ struct FwdLayout {
   Sched lse_sched;
   int K, M;   // heads, rows of the unembedding GEMM
   bool wide;  // the unembedding runs on 256-row tiles
+  int parts;  // (max, sum-exp) partials per logit row: one per vocabulary range
 };
 
 FwdLayout fwd_layout(const cpmtp_shape& s, int sms) {
@@ -164,6 +200,7 @@ FwdLayout fwd_layout(const cpmtp_shape& s, int sms) {
   const int m_tiles = (L.M + bm - 1) / bm;
   const int n_tiles = (s.V + kBN - 1) / kBN;
   L.lse_sched = sched_lse(m_tiles, n_tiles, L.M, s.V, s.d, bm, sms);
+  L.parts = L.lse_sched.n_splits;
   size_t off = 0;
   auto take = [&](size_t bytes) { size_t o = off; off = align_up(off + bytes); return o; };
   L.logw = take(sizeof(float) * s.N * s.r);
@@ -173,8 +210,8 @@ FwdLayout fwd_layout(const cpmtp_shape& s, int sms) {
   L.tgt = take(sizeof(float) * L.M);
   L.z = take(2ull * L.M * s.d);
   L.tgt_part = take(sizeof(float) * static_cast<size_t>(L.M) * (s.d / 64));
-  L.part_m = take(sizeof(float) * static_cast<size_t>(L.M) * L.lse_sched.n_splits);
-  L.part_l = take(sizeof(float) * static_cast<size_t>(L.M) * L.lse_sched.n_splits);
+  L.part_m = take(sizeof(float) * static_cast<size_t>(L.M) * L.parts);
+  L.part_l = take(sizeof(float) * static_cast<size_t>(L.M) * L.parts);
   L.total = off;
   return L;
 }
@@ -199,10 +236,18 @@ BwdLayout bwd_layout(const cpmtp_shape& s, int quantum = kBM, bool distill = fal
   L.M = s.N * L.K;
   L.ldg = (s.V + 63) / 64 * 64;
   long long rows = static_cast<long long>(kLogitGradBudgetBytes / (2ull * L.ldg)) / quantum * quantum;
-  if (const char* env = std::getenv("CPMTP_BWD_CHUNK_ROWS")) {
-    const long long v = std::atoll(env);
-    if (v >= quantum) rows = v / quantum * quantum;
+  if (rows < L.M) {
+    // Several chunks: make a chunk a whole number of waves of the dz GEMM (row tiles x d/256 column tiles over
+    // one CTA per SM), whose last wave would otherwise run partly empty in every chunk.
+    const int sms = sms_or_default();
+    const long long tile_rows = use_wide(rows, s.V) ? kWideBM : kBM;
+    const long long col_tiles = (s.d + kBN - 1) / kBN;
+    long long g = sms, b = col_tiles;
+    while (b != 0) { const long long t = g % b; g = b; b = t; }
+    const long long wave_rows = tile_rows * (sms / g);
+    if (rows >= 2 * wave_rows) rows = rows / wave_rows * wave_rows / quantum * quantum;
   }
+  if (knobs().bwd_chunk_rows >= quantum) rows = knobs().bwd_chunk_rows / quantum * quantum;   // testing knob
   if (rows < quantum) rows = quantum;
   const long long m_pad = (static_cast<long long>(L.M) + quantum - 1) / quantum * quantum;
   if (rows > m_pad) rows = m_pad;
@@ -227,7 +272,7 @@ BwdLayout bwd_layout(const cpmtp_shape& s, int quantum = kBM, bool distill = fal
 // Distillation forward: the plain forward pass, then the grouped KL pass over the vocabulary.
 struct DistillLayout {
   FwdLayout fwd;
-  size_t part, total;
+  size_t part, part_tm, part_tl, total;
   Sched sched;
   int R, gpt, groups;   // padded rank, groups per 128-row tile, N * n
 };
@@ -252,9 +297,7 @@ DistillLayout distill_layout(const cpmtp_shape& s, int sms) {
   }
   {
     // tuning knobs for this sweep alone
-    int g = 0, sp = 0;
-    if (const char* env = std::getenv("CPMTP_KL_GROUP_TILES")) g = std::atoi(env);
-    if (const char* env = std::getenv("CPMTP_KL_SPLITS")) sp = std::atoi(env);
+    const int g = static_cast<int>(knobs().kl_group_tiles), sp = static_cast<int>(knobs().kl_splits);
     if (g >= 1 || sp >= 1)
       L.sched = make_sched(m_tiles, n_tiles, sp >= 1 ? sp : L.sched.n_splits, g >= 1 ? g : L.sched.m_group, s.d / kBK);
   }
@@ -262,6 +305,8 @@ DistillLayout distill_layout(const cpmtp_shape& s, int sms) {
   size_t off = align_up(L.fwd.total);
   auto take = [&](size_t bytes) { size_t o = off; off = align_up(off + bytes); return o; };
   L.part = take(sizeof(float) * static_cast<size_t>(L.fwd.M) * L.sched.n_splits);
+  L.part_tm = take(sizeof(float) * static_cast<size_t>(L.groups) * L.sched.n_splits);
+  L.part_tl = take(sizeof(float) * static_cast<size_t>(L.groups) * L.sched.n_splits);
   L.total = off;
   return L;
 }
@@ -336,10 +381,7 @@ FullBwdLayout full_bwd_layout(const cpmtp_shape& s) {
   L.K = s.n * s.r;
   L.ldv = (s.V + 63) / 64 * 64;
   long long heads = static_cast<long long>(kLogitGradBudgetBytes / (2ull * s.N * L.ldv));
-  if (const char* env = std::getenv("CPMTP_BWD_CHUNK_HEADS")) {   // testing knob
-    const long long v = std::atoll(env);
-    if (v >= 1) heads = v;
-  }
+  if (knobs().bwd_chunk_heads >= 1) heads = knobs().bwd_chunk_heads;   // testing knob
   if (heads < 1) heads = 1;
   if (heads > L.K) heads = L.K;
   L.heads_per_chunk = static_cast<int>(heads);
@@ -358,7 +400,7 @@ FullBwdLayout full_bwd_layout(const cpmtp_shape& s) {
 
 struct SampleLayout {
   FwdLayout fwd;
-  size_t logits, z32, lb, part_top, part_best, logp_tmp, total;
+  size_t logits, z32, lb, part_top, part_best, logp_tmp, done, total;
   int lds, chunks;
 };
 
@@ -375,37 +417,126 @@ SampleLayout sample_layout(const cpmtp_shape& s, int sms) {
   L.part_top = take(sizeof(Cand) * static_cast<size_t>(s.N) * L.chunks * kMaxTopk);
   L.part_best = take(sizeof(Cand) * static_cast<size_t>(s.N) * L.chunks);
   L.logp_tmp = take(sizeof(float) * s.N);
+  L.done = take(sizeof(unsigned int) * s.N);   // per-position count of finished blocks in a draft step
   L.total = off;
   return L;
 }
 
+// Tensor maps depend only on (base address, extents, stride, box), so they are encoded once and kept:
+// a decode loop that calls with the same buffers every step does no driver work on the host after the
+// first call.  Small direct-mapped cache; a map never goes stale (it holds no more than its key).
+struct TmapKey {
+  const void* base;
+  uint64_t rows, k, ld;
+  uint32_t box_rows, groups;   // groups > 0: grouped-row 3-D map (box_rows = padded group size)
+  uint32_t mn_major, group_rows;
+  bool operator==(const TmapKey& o) const { return std::memcmp(this, &o, sizeof(TmapKey)) == 0; }
+};
+struct TmapSlot {
+  TmapKey key;
+  CUtensorMap map;
+  bool used = false;
+};
+constexpr int kTmapSlots = 256;
+TmapSlot g_tmaps[kTmapSlots];
+
+bool cached_tmap(CUtensorMap* out, const TmapKey& key) {
+  uint64_t hsh = reinterpret_cast<uintptr_t>(key.base) * 0x9E3779B97F4A7C15ull;
+  hsh ^= (key.rows * 31 + key.k) * 0xC2B2AE3D27D4EB4Full + key.ld * 7 + key.box_rows * 131 + key.groups * 17 + key.mn_major;
+  TmapSlot& slot = g_tmaps[(hsh >> 20) % kTmapSlots];
+  std::lock_guard<std::mutex> lock(g_cache_mutex);
+  if (slot.used && slot.key == key) {
+    *out = slot.map;
+    return true;
+  }
+  CUtensorMap m;
+  const bool ok = key.groups > 0
+                      ? make_grouped_tmap_bf16(&m, key.base, key.k, key.group_rows, key.rows / key.group_rows, key.ld,
+                                               key.box_rows, key.groups)
+                      : make_operand_tmap(&m, key.base, key.mn_major != 0, key.rows, key.k, key.ld, key.box_rows);
+  if (!ok) return false;
+  slot.key = key;
+  slot.map = m;
+  slot.used = true;
+  *out = m;
+  return true;
+}
+
+// Launch with programmatic stream serialization: the kernel may be scheduled while the one before it in
+// the stream drains; it calls ptx::grid_dep_wait() before it touches anything that kernel produced.
+template <class... KArgs, class... Args>
+cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t stream,
+                       Args... args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid;
+  cfg.blockDim = block;
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = stream;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
+}
+
 template <class Cfg, class Epi>
 cudaError_t launch_gemm(const void* A, uint64_t a_rows, uint64_t a_ld, const void* B, uint64_t b_rows,
-                        uint64_t b_ld, uint64_t kdim, const Sched& sched, const typename Epi::Params& ep,
+                        uint64_t b_ld, uint64_t kdim, const Sched& sched_in, const typename Epi::Params& ep,
                         int* dev_status, int sms, cudaStream_t stream, int a_group_rows = 0) {
   static bool attr_set[64] = {};
   CUtensorMap tA, tB;
-  if (sched.a_groups > 0) {
+  TmapKey ka, kb;
+  std::memset(&ka, 0, sizeof(ka));
+  std::memset(&kb, 0, sizeof(kb));
+  ka.base = A; ka.rows = a_rows; ka.k = kdim; ka.ld = a_ld;
+  if (sched_in.a_groups > 0) {
     // grouped rows: a_rows = groups * a_group_rows, every group padded to 128 / a_groups tile rows
     if (Cfg::A_MN || Cfg::MB != 1 || Cfg::A_ROWS != kBM || a_group_rows < 1) return cudaErrorInvalidValue;
-    if (!make_grouped_tmap_bf16(&tA, A, kdim, a_group_rows, a_rows / a_group_rows, a_ld, kBM / sched.a_groups,
-                                sched.a_groups))
-      return cudaErrorInvalidValue;
-  } else if (!make_operand_tmap(&tA, A, Cfg::A_MN, a_rows, kdim, a_ld, Cfg::A_ROWS * Cfg::MB)) {
-    return cudaErrorInvalidValue;
+    ka.box_rows = kBM / sched_in.a_groups; ka.groups = sched_in.a_groups; ka.group_rows = a_group_rows;
+  } else {
+    ka.box_rows = Cfg::A_ROWS * Cfg::MB; ka.mn_major = Cfg::A_MN ? 1 : 0;
   }
-  if (!make_operand_tmap(&tB, B, Cfg::B_MN, b_rows, kdim, b_ld, Cfg::BN)) return cudaErrorInvalidValue;
+  if (!cached_tmap(&tA, ka)) return cudaErrorInvalidValue;
+  kb.base = B; kb.rows = b_rows; kb.k = kdim; kb.ld = b_ld; kb.box_rows = Cfg::BN; kb.mn_major = Cfg::B_MN ? 1 : 0;
+  if (!cached_tmap(&tB, kb)) return cudaErrorInvalidValue;
   constexpr int smem = gemm_smem_bytes<Cfg, Epi>();
   int dev = 0;
   cudaGetDevice(&dev);
-  if (dev >= 0 && dev < 64 && !attr_set[dev]) {
-    cudaError_t e = cudaFuncSetAttribute(tc_gemm_kernel<Cfg, Epi>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
-    if (e != cudaSuccess) return e;
-    attr_set[dev] = true;
+  if (dev >= 0 && dev < 64) {
+    std::lock_guard<std::mutex> lock(g_cache_mutex);
+    if (!attr_set[dev]) {
+      cudaError_t e = cudaFuncSetAttribute(tc_gemm_kernel<Cfg, Epi>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+      if (e != cudaSuccess) return e;
+      attr_set[dev] = true;
+    }
   }
+  Sched sched = sched_in;
+  // every wait inside the kernel gives up after this long (default 4 s; the knob exists so that a test can
+  // watch the give-up path finish in milliseconds)
+  sched.wait_limit_us = knobs().wait_limit_us > 0 ? static_cast<unsigned>(knobs().wait_limit_us) : 4000000u;
+  sched.test_skip_load = static_cast<int>(knobs().test_skip_load);
   const int grid = sched.units < sms ? sched.units : sms;
-  tc_gemm_kernel<Cfg, Epi><<<grid, Cfg::THREADS, smem, stream>>>(tA, tB, sched, ep, dev_status);
-  return cudaGetLastError();
+  return launch_pdl(tc_gemm_kernel<Cfg, Epi>, dim3(grid), dim3(Cfg::THREADS), smem, stream, tA, tB, sched, ep,
+                    dev_status);
+}
+
+// K-major x K-major launch on 128- or 256-row tiles.
+template <class Epi>
+cudaError_t launch_kk(bool wide, const void* A, uint64_t a_rows, uint64_t a_ld, const void* B, uint64_t b_rows,
+                      uint64_t b_ld, uint64_t kdim, const Sched& sched, const typename Epi::Params& ep,
+                      int* dev_status, int sms, cudaStream_t stream) {
+  if (wide) return launch_gemm<WideKK, Epi>(A, a_rows, a_ld, B, b_rows, b_ld, kdim, sched, ep, dev_status, sms, stream);
+  return launch_gemm<CfgKK, Epi>(A, a_rows, a_ld, B, b_rows, b_ld, kdim, sched, ep, dev_status, sms, stream);
+}
+
+// Tensor map of a row-major bf16 output [rows, cols] (row stride ld) written by the epilogues' TMA stores
+// in boxes of 64 columns x 32 rows.
+bool output_tmap(CUtensorMap* out, const void* base, uint64_t rows, uint64_t cols, uint64_t ld) {
+  TmapKey key;
+  std::memset(&key, 0, sizeof(key));
+  key.base = base; key.rows = rows; key.k = cols; key.ld = ld; key.box_rows = 32;
+  return cached_tmap(out, key);
 }
 
 // A plain GEMM D[m_rows, n_cols] = A * B^T over `kdim`, every column tile its own unit, row tiles
@@ -413,14 +544,12 @@ cudaError_t launch_gemm(const void* A, uint64_t a_rows, uint64_t a_ld, const voi
 template <bool A_MN, bool B_MN, class Epi>
 cudaError_t gemm_auto(const void* A, uint64_t a_ld, const void* B, uint64_t b_ld, long long m_rows, int n_cols,
                       long long kdim, int group_rows, const typename Epi::Params& ep, int* dev_status, int sms,
-                      cudaStream_t stream) {
+                      cudaStream_t stream, int force_tile_rows = 0) {
   const int n_tiles = (n_cols + kBN - 1) / kBN;
   const int k_blocks = static_cast<int>((kdim + kBK - 1) / kBK);
-  if (const char* env = std::getenv("CPMTP_GEMM_GROUP_ROWS")) {   // tuning knob
-    const int v = std::atoi(env);
-    if (v >= kWideBM) group_rows = v;
-  }
-  if (use_wide(m_rows, kdim)) {
+  if (knobs().gemm_group_rows >= kWideBM) group_rows = static_cast<int>(knobs().gemm_group_rows);   // tuning knob
+  const bool wide = force_tile_rows == kWideBM ? true : force_tile_rows == kBM ? false : use_wide(m_rows, kdim);
+  if (wide) {
     const int m_tiles = static_cast<int>((m_rows + kWideBM - 1) / kWideBM);
     const Sched sc = make_sched(m_tiles, n_tiles, n_tiles, group_rows / kWideBM, k_blocks);
     return launch_gemm<TileCfg<kBN, kWideStages, A_MN, B_MN, kBM, 2>, Epi>(A, m_rows, a_ld, B, n_cols, b_ld, kdim, sc,
@@ -458,35 +587,33 @@ int run_forward(const cpmtp_shape& s, const uint16_t* h, const uint16_t* W_head,
   // head projection: z[N, K*d] = h[N, d] * W_cat[K*d, d]^T, plus the fp32 target-logit partials
   {
     ProfScope prof(CPMTP_STAGE_PROJ, stream);
-    EpiProj<kBN>::Params ep{z, tgt_part, E, x, z32, dev_status, s.N, ncols, s.d, s.V, s.n, s.r};
+    EpiProj<kBN>::Params ep{{}, z, tgt_part, E, x, z32, dev_status, s.N, ncols, s.d, s.V, s.n, s.r};
+    if (!output_tmap(&ep.z_map, z, s.N, ncols, ncols)) return CPMTP_ERR_LAUNCH;
     if (s.N <= CfgKKSkinny::A_ROWS) {
       const int n_tiles = (ncols + kBN - 1) / kBN;
       const Sched sc = make_sched(1, n_tiles, n_tiles, 1, s.d / kBK);
       CPMTP_TRY((launch_gemm<CfgKKSkinny, EpiProj<kBN>>(h, s.N, s.d, W_head, ncols, s.d, s.d, sc, ep, dev_status, sms, stream)));
     } else {
-      CPMTP_TRY((gemm_auto<false, false, EpiProj<kBN>>(h, s.d, W_head, s.d, s.N, ncols, s.d, 8192, ep, dev_status, sms, stream)));
+      CPMTP_TRY((gemm_auto<false, false, EpiProj<kBN>>(h, s.d, W_head, s.d, s.N, ncols, s.d, 8192, ep, dev_status, sms, stream,
+                                                      static_cast<int>(knobs().proj_tiles))));   // knob: tuning only
     }
   }
   // unembedding fused with the vocabulary log-sum-exp (Eq. 6, Eq. 8)
   {
     ProfScope prof(CPMTP_STAGE_LSE, stream);
     if (logits != nullptr) {
-      EpiLse<kBN, true>::Params ep{part_m, part_l, L.M, s.V, L.lse_sched.n_splits, logits, lds};
+      EpiLse<kBN, true>::Params ep{part_m, part_l, L.M, s.V, L.parts, logits, lds};
       if (L.M <= CfgKKSkinny::A_ROWS) {
         CPMTP_TRY((launch_gemm<CfgKKSkinny, EpiLse<kBN, true>>(z, L.M, s.d, E, s.V, s.d, s.d, L.lse_sched, ep, dev_status, sms, stream)));
-      } else if (L.wide) {
-        CPMTP_TRY((launch_gemm<WideKK, EpiLse<kBN, true>>(z, L.M, s.d, E, s.V, s.d, s.d, L.lse_sched, ep, dev_status, sms, stream)));
       } else {
-        CPMTP_TRY((launch_gemm<CfgKK, EpiLse<kBN, true>>(z, L.M, s.d, E, s.V, s.d, s.d, L.lse_sched, ep, dev_status, sms, stream)));
+        CPMTP_TRY((launch_kk<EpiLse<kBN, true>>(L.wide, z, L.M, s.d, E, s.V, s.d, s.d, L.lse_sched, ep, dev_status, sms, stream)));
       }
     } else {
-      EpiLse<kBN>::Params ep{part_m, part_l, L.M, s.V, L.lse_sched.n_splits, nullptr, 0};
+      EpiLse<kBN>::Params ep{part_m, part_l, L.M, s.V, L.parts, nullptr, 0};
       if (L.M <= CfgKKSkinny::A_ROWS) {
         CPMTP_TRY((launch_gemm<CfgKKSkinny, EpiLse<kBN>>(z, L.M, s.d, E, s.V, s.d, s.d, L.lse_sched, ep, dev_status, sms, stream)));
-      } else if (L.wide) {
-        CPMTP_TRY((launch_gemm<WideKK, EpiLse<kBN>>(z, L.M, s.d, E, s.V, s.d, s.d, L.lse_sched, ep, dev_status, sms, stream)));
       } else {
-        CPMTP_TRY((launch_gemm<CfgKK, EpiLse<kBN>>(z, L.M, s.d, E, s.V, s.d, s.d, L.lse_sched, ep, dev_status, sms, stream)));
+        CPMTP_TRY((launch_kk<EpiLse<kBN>>(L.wide, z, L.M, s.d, E, s.V, s.d, s.d, L.lse_sched, ep, dev_status, sms, stream)));
       }
     }
   }
@@ -494,10 +621,8 @@ int run_forward(const cpmtp_shape& s, const uint16_t* h, const uint16_t* W_head,
   {
     ProfScope prof(CPMTP_STAGE_MIXTURE, stream);
     const int threads = s.N <= 256 ? 1024 : 256;
-    gate_mixture_kernel<<<s.N, threads, 0, stream>>>(h, W_g, s.d, part_m, part_l, L.lse_sched.n_splits, tgt_part,
-                                                    x != nullptr ? s.d / 64 : 0, logw, lse, tgt, q, logp, logp_prefix,
-                                                    s.N, s.n, s.r);
-    CPMTP_TRY(cudaGetLastError());
+    CPMTP_TRY(launch_pdl(gate_mixture_kernel, dim3(s.N), dim3(threads), 0, stream, h, W_g, s.d, part_m, part_l, L.parts,
+                         tgt_part, x != nullptr ? s.d / 64 : 0, logw, lse, tgt, q, logp, logp_prefix, s.N, s.n, s.r));
   }
   if (loss != nullptr || counts != nullptr || saved != nullptr) {
     ProfScope prof(CPMTP_STAGE_FINALIZE, stream);
@@ -546,17 +671,13 @@ static unsigned char* static_scratch_ptr() {
   static unsigned char* ptrs[64] = {};
   int dev = 0;
   if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return nullptr;
+  std::lock_guard<std::mutex> lock(g_cache_mutex);
   if (ptrs[dev] == nullptr) {
     void* p = nullptr;
     if (cudaGetSymbolAddress(&p, g_static_scratch) != cudaSuccess || p == nullptr) return nullptr;
     ptrs[dev] = static_cast<unsigned char*>(p);
   }
   return ptrs[dev];
-}
-
-static int sms_or_default() {
-  DeviceInfo* di = device_info();
-  return (di != nullptr && di->sms > 0) ? di->sms : 148;
 }
 
 
@@ -620,6 +741,7 @@ static int backward_impl(const cpmtp_shape* shape, const void* h, const void* W_
   const int ncols = K * d;
   const float aux = (s.flags & CPMTP_FLAG_AUX) ? s.aux_coef : 0.f;
   const int per_token = (s.flags & CPMTP_FLAG_PER_TOKEN) ? 1 : 0;
+  const int accum = (s.flags & CPMTP_FLAG_ACCUM_GRADS) ? 1 : 0;   // outputs += instead of =
   if (per_token && dloss_dlogp == nullptr && dc == nullptr) return CPMTP_ERR_NULL;
   float* uk = reinterpret_cast<float*>(ws + L.uk);
 
@@ -658,7 +780,8 @@ static int backward_impl(const cpmtp_shape* shape, const void* h, const void* W_
       CPMTP_TRY((launch_grouped<EpiDistillGrad>(R, zc, rows, d, Eb, V, sc, ep, s.r, dev_status, sms, st)));
     } else if (dc == nullptr && (need_dz || dE != nullptr)) {
       ProfScope prof(CPMTP_STAGE_LOGIT_GRAD, st);
-      EpiLogitGrad<kBN>::Params ep{G, saved->lse, coef, x, row0, rows, L.ldg, V, K, s.n, s.r};
+      EpiLogitGrad<kBN>::Params ep{{}, G, saved->lse, coef, x, row0, rows, L.ldg, V, K, s.n, s.r};
+      if (!output_tmap(&ep.G_map, G, rows, L.ldg, L.ldg)) return CPMTP_ERR_LAUNCH;
       CPMTP_TRY((gemm_auto<false, false, EpiLogitGrad<kBN>>(zc, d, Eb, d, rows, V, d, 2048, ep, dev_status, sms, st)));
     }
     // dz[rows, d] = G[rows, V] * E[V, d]
@@ -671,7 +794,7 @@ static int backward_impl(const cpmtp_shape* shape, const void* h, const void* W_
     if (dE != nullptr) {
       ProfScope prof(CPMTP_STAGE_DE, st);
       if (L.chunks == 1) {
-        EpiStoreBf16<kBN, false>::Params ep{static_cast<uint16_t*>(dE), nullptr, nullptr, V, d, d, 0};
+        EpiStoreBf16<kBN, false>::Params ep{static_cast<uint16_t*>(dE), nullptr, nullptr, V, d, d, 0, accum};
         CPMTP_TRY((gemm_auto<true, true, EpiStoreBf16<kBN, false>>(G, L.ldg, zc, d, V, d, rows, 2048, ep, dev_status, sms, st)));
       } else {
         EpiAccumF32<kBN>::Params ep{dE32, V, d, d, c > 0 ? 1 : 0};
@@ -681,19 +804,19 @@ static int backward_impl(const cpmtp_shape* shape, const void* h, const void* W_
   }
   if (L.chunks > 1 && dE != nullptr) {
     ProfScope prof(CPMTP_STAGE_DE_CONVERT, st);
-    f32_to_bf16_kernel<<<sms * 8, 256, 0, st>>>(dE32, static_cast<uint16_t*>(dE), static_cast<size_t>(V) * d);
+    f32_to_bf16_kernel<<<sms * 8, 256, 0, st>>>(dE32, static_cast<uint16_t*>(dE), static_cast<size_t>(V) * d, accum);
     CPMTP_TRY(cudaGetLastError());
   }
   // dW_head[K*d, d] = dz^T[K*d, N] * h[N, d]
   if (dW_head != nullptr) {
     ProfScope prof(CPMTP_STAGE_DW_HEAD, st);
-    EpiStoreBf16<kBN, false>::Params ep{static_cast<uint16_t*>(dW_head), nullptr, nullptr, ncols, d, d, 0};
+    EpiStoreBf16<kBN, false>::Params ep{static_cast<uint16_t*>(dW_head), nullptr, nullptr, ncols, d, d, 0, accum};
     CPMTP_TRY((gemm_auto<true, true, EpiStoreBf16<kBN, false>>(dz, ncols, h, d, ncols, d, s.N, 2048, ep, dev_status, sms, st)));
   }
   // dh[N, d] = dz[N, K*d] * W_cat[K*d, d] + dg * W_g
   if (dh != nullptr) {
     ProfScope prof(CPMTP_STAGE_DH, st);
-    EpiStoreBf16<kBN, true>::Params ep{static_cast<uint16_t*>(dh), dg, static_cast<const uint16_t*>(W_g), s.N, d, d, s.r};
+    EpiStoreBf16<kBN, true>::Params ep{static_cast<uint16_t*>(dh), dg, static_cast<const uint16_t*>(W_g), s.N, d, d, s.r, accum};
     CPMTP_TRY((gemm_auto<false, true, EpiStoreBf16<kBN, true>>(dz, ncols, W_head, d, s.N, d, ncols, 2048, ep, dev_status, sms, st)));
   }
   // dW_g[r, d] = dg^T * h
@@ -704,7 +827,7 @@ static int backward_impl(const cpmtp_shape* shape, const void* h, const void* W_
                                                           L.dwg_rows_per_slice);
     CPMTP_TRY(cudaGetLastError());
     dwg_reduce_kernel<<<(s.r * d + 255) / 256, 256, 0, st>>>(dwg_part, static_cast<uint16_t*>(dW_g), L.dwg_slices,
-                                                            s.r, d);
+                                                            s.r, d, accum);
     CPMTP_TRY(cudaGetLastError());
   }
   return CPMTP_OK;
@@ -713,7 +836,14 @@ static int backward_impl(const cpmtp_shape* shape, const void* h, const void* W_
 
 extern "C" {
 
-int cpmtp_version(void) { return 110; }   // 1.1: distillation entry points
+int cpmtp_version(void) { return 120; }   // 1.2: gradient accumulation flag, knob reload
+
+int cpmtp_reload_knobs(void) {
+  knobs();   // make sure the one-time read has happened, then read again
+  std::lock_guard<std::mutex> lock(g_cache_mutex);
+  read_knobs();
+  return CPMTP_OK;
+}
 
 int cpmtp_profile_begin(void) {
   for (cudaEvent_t e : g_prof.events) cudaEventDestroy(e);
@@ -828,6 +958,7 @@ int cpmtp_sample_draft(const cpmtp_shape* shape, const void* h, const void* W_he
   if (rc != CPMTP_OK) return rc;
   if (draft == nullptr) return CPMTP_ERR_NULL;
   if (topk < 1 || topk > kMaxTopk || topk > shape->V) return CPMTP_ERR_SHAPE;
+  if (shape->N > 65535) return CPMTP_ERR_LIMIT;   // positions ride on gridDim.y
   if (uniform != nullptr && !(temperature > 0.f)) return CPMTP_ERR_SHAPE;
   const cpmtp_shape& s = *shape;
   const SampleLayout L = sample_layout(s, di->sms);
@@ -849,16 +980,13 @@ int cpmtp_sample_draft(const cpmtp_shape* shape, const void* h, const void* W_he
   if (rf != CPMTP_OK) return rf;
   CPMTP_TRY(cudaMemcpyAsync(lb, logw, sizeof(float) * s.N * s.r, cudaMemcpyDeviceToDevice, st));   // b = w
   const float inv_temp = uniform != nullptr ? 1.0f / temperature : 1.0f;
+  unsigned int* done = reinterpret_cast<unsigned int*>(ws + L.done);
+  CPMTP_TRY(cudaMemsetAsync(done, 0, sizeof(unsigned int) * s.N, st));
   for (int step = 0; step < s.n; ++step) {
     ProfScope prof(CPMTP_STAGE_DRAFT_STEP, st);
-    draft_step_partial_kernel<<<dim3(L.chunks, s.N), kSampleThreads, 0, st>>>(
-        logits, L.lds, lse, lb, uniform, inv_temp, step, s.V, s.n, s.r, topk, part_top, part_best);
-    CPMTP_TRY(cudaGetLastError());
-    draft_step_final_kernel<<<s.N, kSampleFinalThreads, 0, st>>>(z32, static_cast<const uint16_t*>(E), s.d, lse, lb,
-                                                           part_top, part_best, L.chunks,
-                                                           uniform != nullptr ? 1 : 0, step, s.V, s.n, s.r, topk,
-                                                           forced, dev_status, draft, logp_joint, topk_tokens,
-                                                           topk_logp);
+    draft_step_kernel<<<dim3(L.chunks, s.N), kSampleThreads, 0, st>>>(
+        logits, L.lds, z32, static_cast<const uint16_t*>(E), s.d, lse, lb, uniform, inv_temp, step, s.V, s.n, s.r,
+        topk, forced, part_top, part_best, done, dev_status, draft, logp_joint, topk_tokens, topk_logp);
     CPMTP_TRY(cudaGetLastError());
   }
   return CPMTP_OK;
@@ -891,11 +1019,7 @@ int cpmtp_forward_full(const cpmtp_shape* shape, const void* h, const void* W_fu
     ProfScope prof(CPMTP_STAGE_LSE, st);
     EpiLseFull<kBN>::Params ep{part_m, part_l, tgt, x, dev_status, s.N, s.V, L.K, s.n, s.r, L.tph, L.K * L.sph};
     const uint64_t b_rows = static_cast<uint64_t>(L.K) * s.V;
-    if (L.wide) {
-      CPMTP_TRY((launch_gemm<WideKK, EpiLseFull<kBN>>(h, s.N, s.d, W_full, b_rows, s.d, s.d, L.sched, ep, dev_status, di->sms, st)));
-    } else {
-      CPMTP_TRY((launch_gemm<CfgKK, EpiLseFull<kBN>>(h, s.N, s.d, W_full, b_rows, s.d, s.d, L.sched, ep, dev_status, di->sms, st)));
-    }
+    CPMTP_TRY((launch_kk<EpiLseFull<kBN>>(L.wide, h, s.N, s.d, W_full, b_rows, s.d, s.d, L.sched, ep, dev_status, di->sms, st)));
   }
   {
     ProfScope prof(CPMTP_STAGE_MIXTURE, st);
@@ -942,6 +1066,7 @@ int cpmtp_backward_full(const cpmtp_shape* shape, const void* h, const void* W_f
   const int K = L.K, d = s.d, V = s.V;
   const float aux = (s.flags & CPMTP_FLAG_AUX) ? s.aux_coef : 0.f;
   const int per_token = (s.flags & CPMTP_FLAG_PER_TOKEN) ? 1 : 0;
+  const int accum = (s.flags & CPMTP_FLAG_ACCUM_GRADS) ? 1 : 0;
   if (per_token && (dloss_dlogp == nullptr || saved->tgt == nullptr)) return CPMTP_ERR_NULL;
   {
     ProfScope prof(CPMTP_STAGE_COEFF, st);
@@ -958,17 +1083,14 @@ int cpmtp_backward_full(const cpmtp_shape* shape, const void* h, const void* W_f
     // recompute the logits of these heads -> G (bf16)
     {
       ProfScope prof(CPMTP_STAGE_LOGIT_GRAD, st);
-      EpiLogitGradFull<kBN>::Params ep{G, saved->lse, coef, x, s.N, V, K, s.n, s.r, tph, L.ldv, ldg, k0};
+      EpiLogitGradFull<kBN>::Params ep{{}, G, saved->lse, coef, x, s.N, V, K, s.n, s.r, tph, L.ldv, ldg, k0};
+      if (!output_tmap(&ep.G_map, G, s.N, ldg, ldg)) return CPMTP_ERR_LAUNCH;
       Sched sc = make_sched((s.N + bm - 1) / bm, heads * tph, heads * tph, 2048 / bm, d / kBK);
       sc.seg_tiles = tph;
       sc.seg_stride = V;
       const uint16_t* Wc = Wf + static_cast<size_t>(k0) * V * d;
       const uint64_t b_rows = static_cast<uint64_t>(heads) * V;
-      if (wide) {
-        CPMTP_TRY((launch_gemm<WideKK, EpiLogitGradFull<kBN>>(hb, s.N, d, Wc, b_rows, d, d, sc, ep, dev_status, sms, st)));
-      } else {
-        CPMTP_TRY((launch_gemm<CfgKK, EpiLogitGradFull<kBN>>(hb, s.N, d, Wc, b_rows, d, d, sc, ep, dev_status, sms, st)));
-      }
+      CPMTP_TRY((launch_kk<EpiLogitGradFull<kBN>>(wide, hb, s.N, d, Wc, b_rows, d, d, sc, ep, dev_status, sms, st)));
     }
     for (int k = k0; k < k0 + heads; ++k) {
       const uint16_t* Gk = G + static_cast<size_t>(k - k0) * L.ldv;
@@ -977,7 +1099,7 @@ int cpmtp_backward_full(const cpmtp_shape* shape, const void* h, const void* W_f
       {
         ProfScope prof(CPMTP_STAGE_DE, st);
         EpiStoreBf16<kBN, false>::Params ep{static_cast<uint16_t*>(dW_full) + static_cast<size_t>(k) * V * d, nullptr,
-                                            nullptr, V, d, d, 0};
+                                            nullptr, V, d, d, 0, accum};
         CPMTP_TRY((gemm_auto<true, true, EpiStoreBf16<kBN, false>>(Gk, ldg, hb, d, V, d, s.N, 2048, ep, dev_status, sms, st)));
       }
       // dh (+)= G_k[N, V] * W_full[k][V, d]
@@ -992,7 +1114,7 @@ int cpmtp_backward_full(const cpmtp_shape* shape, const void* h, const void* W_f
     ProfScope prof(CPMTP_STAGE_DE_CONVERT, st);
     const size_t total = static_cast<size_t>(s.N) * d;
     dh_finish_kernel<<<static_cast<unsigned>((total + 255) / 256), 256, 0, st>>>(
-        dh32, dg, static_cast<const uint16_t*>(W_g), static_cast<uint16_t*>(dh), s.N, d, s.r);
+        dh32, dg, static_cast<const uint16_t*>(W_g), static_cast<uint16_t*>(dh), s.N, d, s.r, accum);
     CPMTP_TRY(cudaGetLastError());
   }
   {
@@ -1000,7 +1122,7 @@ int cpmtp_backward_full(const cpmtp_shape* shape, const void* h, const void* W_f
     dim3 grid((d + 127) / 128, L.dwg_slices);
     dwg_partial_kernel<CPMTP_MAX_R><<<grid, 128, 0, st>>>(dg, hb, dwg_part, s.N, d, s.r, L.dwg_rows_per_slice);
     CPMTP_TRY(cudaGetLastError());
-    dwg_reduce_kernel<<<(s.r * d + 255) / 256, 256, 0, st>>>(dwg_part, static_cast<uint16_t*>(dW_g), L.dwg_slices, s.r, d);
+    dwg_reduce_kernel<<<(s.r * d + 255) / 256, 256, 0, st>>>(dwg_part, static_cast<uint16_t*>(dW_g), L.dwg_slices, s.r, d, accum);
     CPMTP_TRY(cudaGetLastError());
   }
   return CPMTP_OK;
@@ -1027,6 +1149,11 @@ int cpmtp_score_draft_static(const cpmtp_shape* shape, const void* h, const void
                              int32_t* dev_status, cpmtp_stream stream) {
   const int vs = validate_shape(shape);
   if (vs != CPMTP_OK) return vs;
+  // architecture first: on a device without an sm_100a image the symbol lookup below would fail
+  // with a less telling error
+  DeviceInfo* dinfo = device_info();
+  if (dinfo == nullptr) return CPMTP_ERR_LAUNCH;
+  if (dinfo->cc_major != 10) return CPMTP_ERR_ARCH;
   unsigned char* scratch = static_scratch_ptr();
   if (scratch == nullptr) return CPMTP_ERR_LAUNCH;
   DeviceInfo* di = nullptr;
@@ -1057,6 +1184,16 @@ int cpmtp_forward_host(const cpmtp_shape* shape, const void* h_host, const void*
   uint8_t* x_dev = h_dev + align_up(h_bytes);
   uint8_t* logp_dev = x_dev + align_up(x_bytes);
   uint8_t* loss_dev = logp_dev + align_up(4ull * shape->N);
+  {
+    // everything cpmtp_forward would refuse is refused here, before anything is enqueued
+    DeviceInfo* di = nullptr;
+    const int rc = check_common(shape, h_dev, W_head, E, W_g, x_dev, workspace, &di);
+    if (rc != CPMTP_OK) return rc;
+    if (saved != nullptr) {
+      const int rs = check_saved(saved, !(shape->flags & CPMTP_FLAG_RECOMPUTE_Z));
+      if (rs != CPMTP_OK) return rs;
+    }
+  }
   CPMTP_TRY(cudaMemcpyAsync(h_dev, h_host, h_bytes, cudaMemcpyHostToDevice, st));
   CPMTP_TRY(cudaMemcpyAsync(x_dev, x_host, x_bytes, cudaMemcpyHostToDevice, st));
   const int rc = cpmtp_forward(shape, h_dev, W_head, E, W_g, reinterpret_cast<const int32_t*>(x_dev),
@@ -1097,25 +1234,25 @@ int cpmtp_distill_forward(const cpmtp_shape* shape, const void* h, const void* W
   const uint16_t* z = recompute_z ? reinterpret_cast<const uint16_t*>(ws + L.fwd.z)
                                   : static_cast<const uint16_t*>(saved->z);
   {
-    ProfScope prof(CPMTP_STAGE_TEACHER_LSE, st);
-    teacher_lse_kernel<<<L.groups, kTeacherThreads, 0, st>>>(Tb, s.V, dsaved->lse_t);
-    CPMTP_TRY(cudaGetLastError());
+    ProfScope prof(CPMTP_STAGE_TEACHER_LSE, st);   // expert weights per token; the teacher's normaliser comes out of the KL sweep
     distill_pi_kernel<<<(s.N + 127) / 128, 128, 0, st>>>(saved->logw, saved->lse, saved->tgt, dsaved->logpi, s.N, s.n,
                                                         s.r);
     CPMTP_TRY(cudaGetLastError());
   }
   float* part = reinterpret_cast<float*>(ws + L.part);
+  float* part_tm = reinterpret_cast<float*>(ws + L.part_tm);
+  float* part_tl = reinterpret_cast<float*>(ws + L.part_tl);
   {
     ProfScope prof(CPMTP_STAGE_KL, st);
-    const KlParams ep{part, saved->lse, dsaved->logpi, dsaved->lse_t, Tb, L.groups, s.r, s.V, L.sched.n_splits,
+    const KlParams ep{part, part_tm, part_tl, saved->lse, dsaved->logpi, Tb, L.groups, s.r, s.V, L.sched.n_splits,
                       s.V % 8 == 0 ? 1 : 0};
     CPMTP_TRY((launch_grouped<EpiKl>(L.R, z, L.fwd.M, s.d, static_cast<const uint16_t*>(E), s.V, L.sched, ep, s.r,
                                      dev_status, di->sms, st)));
   }
   {
     ProfScope prof(CPMTP_STAGE_FINALIZE, st);
-    distill_merge_kernel<<<(L.groups + 3) / 4, 128, 0, st>>>(part, L.sched.n_splits, dsaved->pm, dsaved->kl, L.groups,
-                                                            s.r);
+    distill_merge_kernel<<<(L.groups + 3) / 4, 128, 0, st>>>(part, part_tm, part_tl, dsaved->logpi, L.sched.n_splits,
+                                                            dsaved->lse_t, dsaved->pm, dsaved->kl, L.groups, s.r);
     CPMTP_TRY(cudaGetLastError());
     if (loss != nullptr) {
       const float aux = (s.flags & CPMTP_FLAG_AUX) ? s.aux_coef : 0.f;

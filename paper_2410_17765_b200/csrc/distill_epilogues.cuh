@@ -60,9 +60,12 @@ struct GroupLanes {
 // p^d on entry and l on exit.  Columns beyond V, rows beyond the last group and a p^d below the
 // smallest normal float (every term underflowed; its weight in the sums is negligible too) give l = 0.
 // vec: V % 8 == 0, so the teacher row is 16-byte aligned and pieces of <= 8 columns never straddle V.
-template <int W>
+// STATS: also fold the teacher logits read here into a running (max, sum-exp) in the log2 domain, so
+// that the teacher's logsumexp needs no pass of its own.
+template <int W, bool STATS = false>
 __device__ __forceinline__ void finish_columns(float* pd, const uint16_t* __restrict__ trow, int col, int V,
-                                               bool row_ok, bool vec, float lse_t) {
+                                               bool row_ok, bool vec, float lse_t, float* tm2 = nullptr,
+                                               float* tl = nullptr) {
   constexpr int P = W < 8 ? W : 8;
 #pragma unroll
   for (int q = 0; q < W / P; ++q) {
@@ -91,6 +94,21 @@ __device__ __forceinline__ void finish_columns(float* pd, const uint16_t* __rest
           if (c + i < V) t[i] = __uint_as_float(static_cast<uint32_t>(__ldg(trow + c + i)) << 16);
       }
     }
+    if constexpr (STATS) {
+      if (row_ok && c < V) {
+        float cm = -INFINITY;
+#pragma unroll
+        for (int i = 0; i < P; ++i)
+          if (c + i < V) cm = fmaxf(cm, t[i]);
+        const float m_new = fmaxf(*tm2, cm * kLog2e);
+        float sum = 0.f;
+#pragma unroll
+        for (int i = 0; i < P; ++i)
+          if (c + i < V) sum += ptx::ex2_approx(fmaf(t[i], kLog2e, -m_new));
+        *tl = *tl * ptx::ex2_approx(*tm2 - m_new) + sum;
+        *tm2 = m_new;
+      }
+    }
 #pragma unroll
     for (int i = 0; i < P; ++i) {
       const float p = pd[q * P + i];
@@ -103,20 +121,24 @@ __device__ __forceinline__ void finish_columns(float* pd, const uint16_t* __rest
 // ---------------------------------------------------------------------------
 // Forward: pm[(g, a)] = sum_v e(v) l(v) with e = pi_{g,a} P^(k)(v | a); the KL term of Eq. 14 for
 // group g is sum_a pm[(g, a)].  One partial per (row, split); rows are ORIGINAL rows g * r + a.
+// The teacher's normaliser logsumexp_v T is not known during the sweep; it enters l(v) as a constant, and
+// sum_v e(v) = pi, so the sweep accumulates  pm' = sum_v e(v) (log p^d(v) - T(v))  together with the running
+// (max, sum-exp) of the teacher logits it reads anyway, and the merge kernel finishes  pm = pm' + pi * lse_t.
+// Every teacher element is therefore read exactly once.
 struct KlParams {
-  float* part;            // [groups * r, splits]
+  float* part;            // [groups * r, splits]  pm' partials
+  float* part_tm;         // [groups, splits]      running max of T * log2(e)
+  float* part_tl;         // [groups, splits]      sum 2^(T * log2(e) - max)
   const float* lse;       // [groups * r]  logsumexp_v S
   const float* logpi;     // [groups * r]  log pi
-  const float* lse_t;     // [groups]      logsumexp_v T
   const uint16_t* T;      // [groups, V]   teacher logits, bf16
   int groups, r, V, splits, vec;
 };
 
 template <int BN, int R>
-struct EpiKl {
+struct EpiKl : EpiDefaults {
   using Params = KlParams;
-  struct State { float c2, lt, acc; long long orow; int grp; bool valid, grp_ok; };
-  static constexpr int SMEM_BYTES = 0;
+  struct State { float c2, tm2, tl, acc; long long orow; int grp; bool valid, grp_ok; };
   using GL = GroupLanes<R>;
   __device__ static void unit_begin(const Params& p, State& st, int m_tile, int, int row_in_tile) {
     st.grp = m_tile * (kBM / R) + row_in_tile / R;
@@ -125,11 +147,23 @@ struct EpiKl {
     st.valid = st.grp_ok && a < p.r;
     st.orow = static_cast<long long>(st.grp) * p.r + a;
     st.c2 = st.valid ? (p.logpi[st.orow] - p.lse[st.orow]) * kLog2e : -INFINITY;
-    st.lt = st.grp_ok ? p.lse_t[st.grp] : 0.f;
+    st.tm2 = -INFINITY;
+    st.tl = 0.f;
     st.acc = 0.f;
   }
-  __device__ static void unit_end(const Params& p, State& st, int, int split, int, uint8_t*, int) {
+  __device__ static void unit_end(const Params& p, State& st, int, int split, int row_in_tile, uint8_t*, int) {
     if (st.valid) p.part[static_cast<size_t>(st.orow) * p.splits + split] = st.acc;
+    // teacher statistics: every lane of the group holds those of its own columns; combine over the group
+    float m = st.tm2;
+#pragma unroll
+    for (int o = R >> 1; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
+    float l = st.tl > 0.f ? st.tl * ptx::ex2_approx(st.tm2 - m) : 0.f;
+#pragma unroll
+    for (int o = R >> 1; o > 0; o >>= 1) l += __shfl_xor_sync(0xffffffffu, l, o);
+    if (st.grp_ok && row_in_tile % R == 0) {
+      p.part_tm[static_cast<size_t>(st.grp) * p.splits + split] = m;
+      p.part_tl[static_cast<size_t>(st.grp) * p.splits + split] = l;
+    }
   }
   __device__ static void tile(const Params& p, State& st, uint32_t tacc, int, int n_tile, int row_in_tile,
                               uint8_t*, int) {
@@ -152,7 +186,7 @@ struct EpiKl {
 #pragma unroll
       for (int j = 0; j < 32; ++j) w[j] = e[j];
       GL::reduce_scatter(w, sub);
-      finish_columns<GL::W>(w, trow, col0 + sub * GL::W, p.V, st.grp_ok, p.vec != 0, st.lt);
+      finish_columns<GL::W, true>(w, trow, col0 + sub * GL::W, p.V, st.grp_ok, p.vec != 0, 0.f, &st.tm2, &st.tl);
       GL::all_gather(w, sub);
       float sum = 0.f;
 #pragma unroll
@@ -181,10 +215,9 @@ struct DistillGradParams {
 };
 
 template <int BN, int R>
-struct EpiDistillGrad {
+struct EpiDistillGrad : EpiDefaults {
   using Params = DistillGradParams;
   struct State { float lse2, pi, coef, ukpi, ckm, lt; long long grp, orow_local; int tok; bool valid, grp_ok; };
-  static constexpr int SMEM_BYTES = 0;
   using GL = GroupLanes<R>;
   __device__ static void unit_begin(const Params& p, State& st, int m_tile, int, int row_in_tile) {
     const int gl = m_tile * (kBM / R) + row_in_tile / R;

@@ -12,39 +12,6 @@ __device__ __forceinline__ float bf16_at(const uint16_t* p, size_t i) {
   return __uint_as_float(static_cast<uint32_t>(__ldg(p + i)) << 16);
 }
 
-// lse_t[g] = logsumexp_v T[g, v]: one block per (position, token) row of the teacher logits.
-constexpr int kTeacherThreads = 256;
-__global__ void __launch_bounds__(kTeacherThreads) teacher_lse_kernel(const uint16_t* __restrict__ T, int V,
-                                                                      float* __restrict__ lse_t) {
-  __shared__ float red[kTeacherThreads / 32];
-  __shared__ float bcast;
-  const uint16_t* row = T + static_cast<size_t>(blockIdx.x) * V;
-  const int t = threadIdx.x, warp = t >> 5, lane = t & 31;
-  float m = -INFINITY;
-  for (int v = t; v < V; v += kTeacherThreads) m = fmaxf(m, bf16_at(row, v));
-  m = warp_max(m);
-  if (lane == 0) red[warp] = m;
-  __syncthreads();
-  if (t == 0) {
-    float mm = red[0];
-    for (int w = 1; w < kTeacherThreads / 32; ++w) mm = fmaxf(mm, red[w]);
-    bcast = mm;
-  }
-  __syncthreads();
-  m = bcast;
-  float l = 0.f;
-  for (int v = t; v < V; v += kTeacherThreads) l += __expf(bf16_at(row, v) - m);
-  l = warp_sum(l);
-  __syncthreads();
-  if (lane == 0) red[warp] = l;
-  __syncthreads();
-  if (t == 0) {
-    float ll = 0.f;
-    for (int w = 0; w < kTeacherThreads / 32; ++w) ll += red[w];
-    lse_t[blockIdx.x] = m + logf(ll);
-  }
-}
-
 // log pi[i, s, a]: the expert weights before token s, pi proportional to w_a prod_{t<s} P^(t)(x_t | a)
 // (sampling section, teacher-forced on the sequence's own tokens).  One thread per position.
 __global__ void distill_pi_kernel(const float* __restrict__ logw, const float* __restrict__ lse,
@@ -68,18 +35,33 @@ __global__ void distill_pi_kernel(const float* __restrict__ logw, const float* _
   }
 }
 
-// pm[row] = sum over splits of the partials; kl[g] = sum_a pm[(g, a)].  One warp per group.
-__global__ void distill_merge_kernel(const float* __restrict__ part, int splits, float* __restrict__ pm,
-                                     float* __restrict__ kl, int groups, int r) {
+// One warp per group g = (position, token).  The teacher's normaliser from the sweep's per-split statistics,
+//   lse_t[g] = logsumexp_v T[g, v]  (two-pass merge of (max, sum-exp) in the log2 domain),
+// then  pm[row] = sum over splits of the pm' partials + pi[row] * lse_t[g]  and  kl[g] = sum_a pm[(g, a)].
+__global__ void distill_merge_kernel(const float* __restrict__ part, const float* __restrict__ part_tm,
+                                     const float* __restrict__ part_tl, const float* __restrict__ logpi, int splits,
+                                     float* __restrict__ lse_t, float* __restrict__ pm, float* __restrict__ kl,
+                                     int groups, int r) {
   const int g = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
   const int lane = threadIdx.x & 31;
   if (g >= groups) return;
+  float m = -INFINITY;
+  for (int j = lane; j < splits; j += 32) m = fmaxf(m, part_tm[static_cast<size_t>(g) * splits + j]);
+  m = warp_max(m);
+  float l = 0.f;
+  for (int j = lane; j < splits; j += 32) {
+    const float lj = part_tl[static_cast<size_t>(g) * splits + j];
+    if (lj > 0.f) l += lj * exp2f(part_tm[static_cast<size_t>(g) * splits + j] - m);
+  }
+  l = warp_sum(l);
+  const float lt = (m + log2f(l)) * 0.6931471805599453f;
+  if (lane == 0) lse_t[g] = lt;
   float total = 0.f;
   for (int a = 0; a < r; ++a) {
     const size_t row = static_cast<size_t>(g) * r + a;
     float v = 0.f;
     for (int j = lane; j < splits; j += 32) v += part[row * splits + j];
-    v = warp_sum(v);
+    v = warp_sum(v) + expf(logpi[row]) * lt;
     if (lane == 0) pm[row] = v;
     total += v;
   }

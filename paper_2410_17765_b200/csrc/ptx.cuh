@@ -48,13 +48,11 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
   return ok != 0;
 }
 
-// Longest time any single wait may take before the CTA gives up (nanoseconds).
-constexpr uint64_t kWaitLimitNs = 4000000000ull;
-
-// Bounded wait.  `abort_flag` lives in shared memory; once any thread of the CTA
-// sets it, every wait that honours it returns false at its next check.
+// Bounded wait: gives up after `limit_ns` nanoseconds (the longest any single wait may take before
+// the CTA unwinds).  `abort_flag` lives in shared memory; once any thread of the CTA sets it, every
+// wait that honours it returns false at its next check.
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag,
-                                          bool honour_abort = true) {
+                                          uint64_t limit_ns, bool honour_abort = true) {
   if (mbar_try_wait(bar, parity)) return true;
   uint32_t spins = 0;
   uint64_t t0 = 0;
@@ -65,7 +63,7 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
       const uint64_t now = globaltimer_ns();
       if (t0 == 0) {
         t0 = now;
-      } else if (now - t0 > kWaitLimitNs) {
+      } else if (now - t0 > limit_ns) {
         *abort_flag = 1;
         return false;
       }
@@ -99,6 +97,24 @@ __device__ __forceinline__ void tma_load_3d(uint32_t smem_dst, const void* tmap,
       : "r"(smem_dst), "l"(reinterpret_cast<uint64_t>(tmap)), "r"(bar), "r"(c0), "r"(c1), "r"(c2)
       : "memory");
 }
+
+// 2-D tiled store, this CTA's shared memory -> global, tracked by the issuing thread's bulk async-group.
+// c0 * element size must be a multiple of 16 B and neither coordinate may be negative; elements of the
+// box that fall outside the tensor are not written.
+__device__ __forceinline__ void tma_store_2d(const void* tmap, uint32_t smem_src, int32_t c0, int32_t c1) {
+  asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%2, %3}], [%1];"
+               :
+               : "l"(reinterpret_cast<uint64_t>(tmap)), "r"(smem_src), "r"(c0), "r"(c1)
+               : "memory");
+}
+__device__ __forceinline__ void bulk_commit_group() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
+// Wait until at most N of this thread's bulk groups still read their shared-memory source.
+template <int N>
+__device__ __forceinline__ void bulk_wait_group_read() {
+  asm volatile("cp.async.bulk.wait_group.read %0;" ::"n"(N) : "memory");
+}
+// Wait until all of this thread's bulk groups have completed (writes performed).
+__device__ __forceinline__ void bulk_wait_group_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
 
 // ----------------------------------------------------------------- tcgen05
 __device__ __forceinline__ void tmem_alloc(uint32_t smem_result_addr, uint32_t ncols) {
@@ -157,6 +173,21 @@ __device__ __forceinline__ void tmem_ld_32x32(uint32_t taddr, float (&v)[32]) {
       : "r"(taddr)
       : "memory");
 }
+// Wait for this thread's outstanding TMEM loads, naming the registers they fill: a tcgen05.ld
+// completes asynchronously, so between its issue and the wait the destination registers hold
+// nothing yet.  Passing them through the wait as read-write operands makes every later use of `v`
+// depend on the wait, whatever the compiler schedules or copies in between.
+__device__ __forceinline__ void tmem_ld_wait_for(float (&v)[32]) {
+  uint32_t* r = reinterpret_cast<uint32_t*>(v);
+  asm volatile(
+      "tcgen05.wait::ld.sync.aligned;"
+      : "+r"(r[0]), "+r"(r[1]), "+r"(r[2]), "+r"(r[3]), "+r"(r[4]), "+r"(r[5]), "+r"(r[6]), "+r"(r[7]),
+        "+r"(r[8]), "+r"(r[9]), "+r"(r[10]), "+r"(r[11]), "+r"(r[12]), "+r"(r[13]), "+r"(r[14]), "+r"(r[15]),
+        "+r"(r[16]), "+r"(r[17]), "+r"(r[18]), "+r"(r[19]), "+r"(r[20]), "+r"(r[21]), "+r"(r[22]), "+r"(r[23]),
+        "+r"(r[24]), "+r"(r[25]), "+r"(r[26]), "+r"(r[27]), "+r"(r[28]), "+r"(r[29]), "+r"(r[30]), "+r"(r[31])
+      :
+      : "memory");
+}
 __device__ __forceinline__ void tmem_ld_32x16(uint32_t taddr, float (&v)[16]) {
   uint32_t* r = reinterpret_cast<uint32_t*>(v);
   asm volatile(
@@ -194,6 +225,15 @@ __host__ __device__ constexpr uint32_t make_idesc_bf16(int M, int N, int a_mn_ma
          (static_cast<uint32_t>(b_mn_major) << 16) | (static_cast<uint32_t>(N >> 3) << 17) |
          (static_cast<uint32_t>(M >> 4) << 24);
 }
+
+// ------------------------------------------- programmatic dependent launch
+// A kernel launched with programmatic stream serialization may start while the kernel before it
+// in the stream is still running.  grid_dep_wait() returns once that kernel has completed and its
+// writes are visible (a no-op in an ordinary launch); everything that reads or overwrites data
+// the previous kernel touches comes after it.  grid_dep_launch() lets the next kernel's blocks be
+// scheduled as soon as every block of this grid has called it or exited.
+__device__ __forceinline__ void grid_dep_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void grid_dep_launch() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 
 // ------------------------------------------------------------------ misc
 __device__ __forceinline__ float ex2_approx(float x) {

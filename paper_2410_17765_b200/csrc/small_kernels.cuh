@@ -67,6 +67,9 @@ __global__ void gate_mixture_kernel(const uint16_t* __restrict__ h, const uint16
       if (lane == 0) g_s[a] = acc;
     }
   }
+  // The gate above reads only the caller's inputs; the partial results below come from the kernel before
+  // this one in the stream (see ptx::grid_dep_wait).
+  ptx::grid_dep_wait();
   // phase 2: per-head vocabulary logsumexp and target logit
   for (int k = warp; k < K; k += nwarps) {
     const size_t row = static_cast<size_t>(i) * K + k;
@@ -281,32 +284,41 @@ __global__ void dwg_partial_kernel(const float* __restrict__ dg, const uint16_t*
   for (int b = 0; b < R_MAX; ++b)
     if (b < r) part[(static_cast<size_t>(slice) * r + b) * d + col] = acc[b];
 }
-// Stage 2: sum the slices in order and round to bf16.
+// Stage 2: sum the slices in order (on top of the stored value when accumulating) and round to bf16.
 __global__ void dwg_reduce_kernel(const float* __restrict__ part, uint16_t* __restrict__ dW_g, int slices,
-                                  int r, int d) {
+                                  int r, int d, int accumulate) {
   const int idx = blockIdx.x * blockDim.x + threadIdx.x;
   if (idx >= r * d) return;
-  float acc = 0.f;
+  float acc = accumulate ? __uint_as_float(static_cast<uint32_t>(dW_g[idx]) << 16) : 0.f;
   for (int s = 0; s < slices; ++s) acc += part[static_cast<size_t>(s) * r * d + idx];
   dW_g[idx] = static_cast<uint16_t>(ptx::pack_bf16x2(acc, 0.f) & 0xFFFFu);
 }
 
 // dh[i, :] = bf16( acc[i, :] + sum_b dg[i, b] * W_g[b, :] ): the gate path of Eq. 7 added to an fp32 sum.
 __global__ void dh_finish_kernel(const float* __restrict__ acc, const float* __restrict__ dg,
-                                 const uint16_t* __restrict__ W_g, uint16_t* __restrict__ dh, int N, int d, int r) {
+                                 const uint16_t* __restrict__ W_g, uint16_t* __restrict__ dh, int N, int d, int r,
+                                 int accumulate) {
   const size_t idx = static_cast<size_t>(blockIdx.x) * blockDim.x + threadIdx.x;
   if (idx >= static_cast<size_t>(N) * d) return;
   const int i = static_cast<int>(idx / d), j = static_cast<int>(idx - static_cast<size_t>(i) * d);
   float v = acc[idx];
+  if (accumulate) v += __uint_as_float(static_cast<uint32_t>(dh[idx]) << 16);
   for (int b = 0; b < r; ++b)
     v = fmaf(dg[static_cast<size_t>(i) * r + b], __uint_as_float(static_cast<uint32_t>(W_g[static_cast<size_t>(b) * d + j]) << 16), v);
   dh[idx] = static_cast<uint16_t>(ptx::pack_bf16x2(v, 0.f) & 0xFFFFu);
 }
 
-__global__ void f32_to_bf16_kernel(const float* __restrict__ src, uint16_t* __restrict__ dst, size_t count) {
+// dst = bf16(src), or bf16(src + dst) when accumulating.  count % 4 == 0.
+__global__ void f32_to_bf16_kernel(const float* __restrict__ src, uint16_t* __restrict__ dst, size_t count,
+                                   int accumulate) {
   const size_t stride = static_cast<size_t>(gridDim.x) * blockDim.x * 4;
   for (size_t i = (static_cast<size_t>(blockIdx.x) * blockDim.x + threadIdx.x) * 4; i < count; i += stride) {
-    const float4 v = *reinterpret_cast<const float4*>(src + i);
+    float4 v = *reinterpret_cast<const float4*>(src + i);
+    if (accumulate) {
+      const uint2 old = *reinterpret_cast<const uint2*>(dst + i);
+      v.x += ptx::bf16_lo(old.x); v.y += ptx::bf16_hi(old.x);
+      v.z += ptx::bf16_lo(old.y); v.w += ptx::bf16_hi(old.y);
+    }
     uint2 o;
     o.x = ptx::pack_bf16x2(v.x, v.y);
     o.y = ptx::pack_bf16x2(v.z, v.w);

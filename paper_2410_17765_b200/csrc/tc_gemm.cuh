@@ -6,7 +6,7 @@
 //   warp 0      TMA producer (one lane): global -> 128B-swizzled shared tiles
 //   warp 1      MMA issuer (one lane): tcgen05.mma, accumulators in TMEM
 //   then 4 epilogue warps per 128-row block: tcgen05.ld the 128 x BN fp32 block and
-//   hand it to `Epi`
+//   hand it to `Epi` (a warp may read only the TMEM lane quarter given by warp id % 4)
 // MB = 1: a 128 x BN tile, accumulator double-buffered in TMEM (2 x BN columns) so the
 //   epilogue of tile j overlaps the MMAs of tile j+1; ring slots of (128 x 64) A + (BN x 64) B.
 // MB = 2 ("wide"): a 256 x 256 tile as two 128-row blocks that share every B slot (two MMAs
@@ -57,6 +57,12 @@ struct Sched {
   // Grouped rows of A (0 = off; K-major A, MB = 1 only): the A tensor map is 3-D [groups][r][K] and a
   // row tile holds a_groups whole groups, each padded to 128 / a_groups rows (see make_grouped_tmap_bf16).
   int a_groups;
+  // Longest time (microseconds) any single wait inside the kernel may take before the CTA gives up,
+  // raises device status 2 and unwinds.  Set by the launcher.
+  unsigned wait_limit_us;
+  // Test hook for that give-up path (0 = off): the producer of every CTA leaves out the load (and the
+  // barrier arrival) of its test_skip_load-th pipeline slot fill, so the consumer's wait for it runs out.
+  int test_skip_load;
 };
 
 inline Sched make_sched(int m_tiles, int n_tiles, int n_splits, int m_group, int k_blocks) {
@@ -74,6 +80,8 @@ inline Sched make_sched(int m_tiles, int n_tiles, int n_splits, int m_group, int
   s.seg_tiles = 0;
   s.seg_stride = 0;
   s.a_groups = 0;
+  s.wait_limit_us = 4000000u;
+  s.test_skip_load = 0;
   return s;
 }
 
@@ -127,20 +135,27 @@ constexpr int kBarrierBytes = 256;
 
 template <class Cfg, class Epi>
 constexpr int gemm_smem_bytes() {
-  return 1024 + Cfg::STAGES * Cfg::STAGE_BYTES + kBarrierBytes + Epi::SMEM_BYTES;
+  return 1024 + Cfg::STAGES * Cfg::STAGE_BYTES + kBarrierBytes + Epi::SMEM_PER_WARP * 4 * Cfg::MB;
 }
 
+// Shared memory: [<= 1023 B alignment pad][STAGES operand slots][epilogue staging: Epi::SMEM_PER_WARP bytes for each
+// of the 4 * MB epilogue warps][barriers].
 template <class Cfg, class Epi>
 __global__ void __launch_bounds__(Cfg::THREADS, 1)
 tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
-               const Sched sched, const typename Epi::Params ep, int* __restrict__ dev_status) {
+               const Sched sched, const __grid_constant__ typename Epi::Params ep, int* __restrict__ dev_status) {
+  constexpr int kEpiSmem = Epi::SMEM_PER_WARP * 4 * Cfg::MB;
+  static_assert(kEpiSmem % 1024 == 0, "epilogue staging keeps the 1024-byte alignment of the slots");
+  static_assert(1024 + Cfg::STAGES * Cfg::STAGE_BYTES + kBarrierBytes + kEpiSmem <= 232448,
+                "more shared memory than a CTA can have");
   extern __shared__ uint8_t smem_raw[];
   const uint32_t raw_addr = ptx::smem_u32(smem_raw);
   const uint32_t pad = (1024u - (raw_addr & 1023u)) & 1023u;
   uint8_t* smem = smem_raw + pad;
   const uint32_t tiles_addr = raw_addr + pad;
-  uint8_t* bar_mem = smem + Cfg::STAGES * Cfg::STAGE_BYTES;
-  const uint32_t bar_addr = tiles_addr + Cfg::STAGES * Cfg::STAGE_BYTES;
+  uint8_t* epi_smem = smem + Cfg::STAGES * Cfg::STAGE_BYTES;
+  uint8_t* bar_mem = epi_smem + kEpiSmem;
+  const uint32_t bar_addr = tiles_addr + Cfg::STAGES * Cfg::STAGE_BYTES + kEpiSmem;
   // barrier layout (8 bytes each): full[STAGES], empty[STAGES], tfull[2], tempty[2], drain
   auto full_bar = [&](int s) { return bar_addr + 8u * s; };
   auto empty_bar = [&](int s) { return bar_addr + 8u * (Cfg::STAGES + s); };
@@ -150,10 +165,10 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
   static_assert(8 * (2 * Cfg::STAGES + 5) + 16 <= kBarrierBytes, "barrier area too small");
   volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(bar_mem + kBarrierBytes - 16);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(bar_mem + kBarrierBytes - 8);
-  uint8_t* epi_smem = bar_mem + kBarrierBytes;
 
   const int warp = threadIdx.x >> 5;
   const int lane = threadIdx.x & 31;
+  const uint64_t wait_ns = static_cast<uint64_t>(sched.wait_limit_us) * 1000ull;
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < Cfg::STAGES; ++s) {
@@ -178,6 +193,9 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
   __syncthreads();
   ptx::tc_fence_after_sync();
   const uint32_t tmem_base = *tmem_slot;
+  // Everything above touched only this CTA's shared memory and TMEM, so it may overlap the tail of the
+  // previous kernel in the stream; the operands and outputs may not.
+  ptx::grid_dep_wait();
 
   if (warp == 0) {
     // ------------------------------------------------------------ producer
@@ -194,7 +212,8 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
           for (int kb = 0; kb < sched.k_blocks; ++kb, ++it) {
             const int s = it % Cfg::STAGES;
             const uint32_t ph = (it / Cfg::STAGES) & 1;
-            if (!ptx::mbar_wait(empty_bar(s), ph ^ 1u, abort_flag)) { alive = false; break; }
+            if (!ptx::mbar_wait(empty_bar(s), ph ^ 1u, abort_flag, wait_ns)) { alive = false; break; }
+            if (sched.test_skip_load != 0 && it + 1 == sched.test_skip_load) continue;   // test hook, see Sched
             ptx::mbar_arrive_expect_tx(full_bar(s), Cfg::STAGE_BYTES);
             const uint32_t a_dst = tiles_addr + s * Cfg::STAGE_BYTES;
             const uint32_t b_dst = a_dst + Cfg::A_BYTES;
@@ -220,11 +239,14 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
           }
         }
       }
+      // All of this CTA's operand loads are issued: the next kernel in the stream may be scheduled
+      // (its blocks start as SMs free up and do their own set-up before they wait for this grid).
+      ptx::grid_dep_launch();
       // Drain: every load issued must have landed before this CTA's shared memory is released.
       const int issued = it;
       for (int back = 1; back <= Cfg::STAGES && back <= issued; ++back) {
         const int j = issued - back;
-        ptx::mbar_wait(full_bar(j % Cfg::STAGES), (j / Cfg::STAGES) & 1, abort_flag, false);
+        ptx::mbar_wait(full_bar(j % Cfg::STAGES), (j / Cfg::STAGES) & 1, abort_flag, wait_ns, false);
       }
     }
   } else if (warp == 1) {
@@ -245,13 +267,13 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         for (int nt = n_begin; nt < n_end && alive; ++nt, ++acc_it) {
           const int acc = acc_it % Cfg::ACC_STAGES;
           const uint32_t acc_ph = (acc_it / Cfg::ACC_STAGES) & 1;
-          if (!ptx::mbar_wait(tempty_bar(acc), acc_ph ^ 1u, abort_flag)) { alive = false; break; }
+          if (!ptx::mbar_wait(tempty_bar(acc), acc_ph ^ 1u, abort_flag, wait_ns)) { alive = false; break; }
           ptx::tc_fence_after_sync();
           const uint32_t d_tmem = tmem_base + acc * Cfg::BN * Cfg::MB;
           for (int kb = 0; kb < sched.k_blocks; ++kb, ++it) {
             const int s = it % Cfg::STAGES;
             const uint32_t ph = (it / Cfg::STAGES) & 1;
-            if (!ptx::mbar_wait(full_bar(s), ph, abort_flag)) { alive = false; break; }
+            if (!ptx::mbar_wait(full_bar(s), ph, abort_flag, wait_ns)) { alive = false; break; }
             ptx::tc_fence_after_sync();
             const uint32_t a_src = tiles_addr + s * Cfg::STAGE_BYTES;
             const uint32_t b_src = a_src + Cfg::A_BYTES;
@@ -272,7 +294,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
       }
       // Drain: all issued MMAs must retire before TMEM is freed.
       ptx::umma_commit(drain_bar);
-      ptx::mbar_wait(drain_bar, 0, abort_flag, false);
+      ptx::mbar_wait(drain_bar, 0, abort_flag, wait_ns, false);
     }
   } else {
     // ------------------------------------------------------------ epilogue
@@ -283,6 +305,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     const int mblock = (warp - 2) >> 2;           // which 128-row block of the tile
     const int row_in_tile = quarter * 32 + lane;  // row within that block
     const int epi_tid = (threadIdx.x - 64) & (kEpiThreads - 1);
+    uint8_t* my_smem = epi_smem + mblock * (Epi::SMEM_PER_WARP * 4);   // this row block's staging
     typename Epi::State st;
     int acc_it = 0;
     bool alive = true;
@@ -294,16 +317,18 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
       for (int nt = n_begin; nt < n_end; ++nt, ++acc_it) {
         const int acc = acc_it % Cfg::ACC_STAGES;
         const uint32_t acc_ph = (acc_it / Cfg::ACC_STAGES) & 1;
-        if (!ptx::mbar_wait(tfull_bar(acc), acc_ph, abort_flag, false)) { alive = false; break; }
+        Epi::pre_tile(ep, st, m_block_tile, nt, row_in_tile);
+        if (!ptx::mbar_wait(tfull_bar(acc), acc_ph, abort_flag, wait_ns, false)) { alive = false; break; }
         ptx::tc_fence_after_sync();
         const uint32_t tacc = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16) +
                               (acc * Cfg::MB + mblock) * Cfg::BN;
-        Epi::tile(ep, st, tacc, m_block_tile, nt, row_in_tile, epi_smem, epi_tid);
+        Epi::tile(ep, st, tacc, m_block_tile, nt, row_in_tile, my_smem, epi_tid);
         ptx::tc_fence_before_sync();
         ptx::mbar_arrive(tempty_bar(acc));
       }
-      if (alive) Epi::unit_end(ep, st, m_block_tile, split, row_in_tile, epi_smem, epi_tid);
+      if (alive) Epi::unit_end(ep, st, m_block_tile, split, row_in_tile, my_smem, epi_tid);
     }
+    Epi::role_end(ep, st, my_smem, epi_tid);   // e.g. wait for this thread's asynchronous stores
   }
 
   ptx::tc_fence_before_sync();

@@ -1,7 +1,6 @@
 """GPU parity of the distillation objective (Eq. 14): cpmtp_distill_forward / _backward through the
 C-ABI against the fp64 oracle on the same seeded bf16 inputs.  Tolerances: KL, prefix scores and loss
 within 2e-3; gradient relative L2 error <= 1e-2."""
-import os
 
 import numpy as np
 import pytest
@@ -53,10 +52,7 @@ def run_case(name, beta=0.9, gamma=0.8, aux=None, chunk_rows=None, up=None, uk=N
     saved = binding.Saved.alloc(cshape)
     dsaved = binding.DistillSaved.alloc(cshape)
     st = torch.zeros(1, dtype=torch.int32, device="cuda")
-    old = os.environ.get("CPMTP_BWD_CHUNK_ROWS")
-    try:
-        if chunk_rows is not None:
-            os.environ["CPMTP_BWD_CHUNK_ROWS"] = str(chunk_rows)
+    with binding.knobs(CPMTP_BWD_CHUNK_ROWS=chunk_rows):
         out = binding.distill_forward(*dev, saved, dsaved, beta=beta, gamma=gamma, aux_coef=aux, dev_status=st,
                                       recompute_z=recompute_z)
         g = binding.distill_backward(*dev, saved, dsaved, beta=beta, gamma=gamma, aux_coef=aux, dev_status=st,
@@ -64,11 +60,6 @@ def run_case(name, beta=0.9, gamma=0.8, aux=None, chunk_rows=None, up=None, uk=N
                                      dloss_dkl=None if uk is None else torch.from_numpy(uk).float().cuda(),
                                      recompute_z=recompute_z, skip=skip)
         torch.cuda.synchronize()
-    finally:
-        if old is None:
-            os.environ.pop("CPMTP_BWD_CHUNK_ROWS", None)
-        else:
-            os.environ["CPMTP_BWD_CHUNK_ROWS"] = old
     assert int(st.item()) == 0
     return inp, T, shape, out, g, dsaved
 

@@ -1,5 +1,4 @@
 """GPU parity of the full-head variant (cpmtp_forward_full / cpmtp_backward_full) against the oracle."""
-import os
 
 import numpy as np
 import pytest
@@ -7,6 +6,7 @@ import torch
 
 from oracle import cp_head
 from paper_2410_17765_b200 import synth
+from parity_checks import assert_expert_counts
 
 pytestmark = pytest.mark.gpu
 
@@ -44,25 +44,17 @@ def test_full_head_forward_and_backward_match_oracle(name, chunk_heads):
     cs = binding.make_shape(shape.N, shape.d, shape.V, shape.n, shape.r)
     saved = binding.Saved.alloc_full(cs)
     st = torch.zeros(1, dtype=torch.int32, device="cuda")
-    old = os.environ.get("CPMTP_BWD_CHUNK_HEADS")
-    try:
-        if chunk_heads is not None:
-            os.environ["CPMTP_BWD_CHUNK_HEADS"] = str(chunk_heads)
+    with binding.knobs(CPMTP_BWD_CHUNK_HEADS=chunk_heads):
         out = binding.forward_full(h, Wf, Wg, x, aux_coef=1.0, saved=saved, want_prefix=True, dev_status=st)
         g = binding.backward_full(h, Wf, Wg, x, saved, aux_coef=1.0, dev_status=st)
         torch.cuda.synchronize()
-    finally:
-        if old is None:
-            os.environ.pop("CPMTP_BWD_CHUNK_HEADS", None)
-        else:
-            os.environ["CPMTP_BWD_CHUNK_HEADS"] = old
     assert int(st.item()) == 0
     assert np.max(np.abs(out["logp"].cpu().numpy() - ref.logp)) <= LOGP_TOL
     assert abs(float(out["loss"].item()) - ref.loss) <= LOGP_TOL
     assert np.max(np.abs(out["logp_prefix"].cpu().numpy() - cp_head.prefix_log_probs(ref))) <= LOGP_TOL
     assert np.max(np.abs(saved.lse.cpu().numpy() - ref.lse)) <= 1e-3
     assert np.max(np.abs(saved.tgt.cpu().numpy() - ref.tgt)) <= 1e-3 * max(1.0, np.abs(ref.tgt).max())
-    assert int(out["counts"].sum().item()) == shape.N
+    assert_expert_counts(out["counts"].cpu().numpy(), ref.logw)
     for key, want in (("dh", refg.dh), ("dW_full", refg.dW_full), ("dW_g", refg.dW_g)):
         got = g[key].float().cpu().numpy()
         if np.linalg.norm(want) == 0:

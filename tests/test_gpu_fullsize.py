@@ -15,6 +15,7 @@ import torch
 
 from oracle import cp_head
 from paper_2410_17765_b200 import synth
+from parity_checks import assert_expert_counts
 
 pytestmark = pytest.mark.gpu
 
@@ -196,7 +197,7 @@ def test_bigvocab_full_size_forward_and_backward_sampled():
     logw = cp_head.gate_log_weights(inp.h, inp.W_g)
     wbar = np.exp(logw).mean(axis=0)
     assert np.max(np.abs(saved.wbar[: s.r].cpu().numpy() - wbar)) <= 1e-5
-    assert int(fwd["counts"].sum().item()) == s.N
+    assert_expert_counts(fwd["counts"].cpu().numpy(), logw)
     loss_ref = -float(fwd["logp"].double().mean().item()) + float(np.sum(wbar ** 2))
     assert abs(float(fwd["loss"].item()) - loss_ref) <= 1e-4
     # gradients: finite, and the hot target rows of dE (Zipf head) are where the mass is
@@ -211,6 +212,49 @@ def test_bigvocab_full_size_forward_and_backward_sampled():
     up = np.full(len(idx), -1.0 / s.N)
     ref = cp_head.backward(sub.h, sub.W_head, sub.E, sub.W_g, sub.x, s.n, s.r, dloss_dlogp=up)
     assert rel_l2(g0["dh"][idx.cuda()].float().cpu().numpy(), ref.dh) <= GRAD_TOL
+
+
+def rel_l2_blocked(got_dev, want):
+    """Relative L2 error of a bf16 device tensor against an fp64 array, one slice of the first axis at a time
+    (the weight gradients at this size are several GB in fp64)."""
+    num = den = 0.0
+    for j in range(want.shape[0]):
+        g = got_dev[j].double().cpu().numpy()
+        num += float(np.sum((g - want[j]) ** 2))
+        den += float(np.sum(want[j] ** 2))
+    return (num / max(den, 1e-300)) ** 0.5
+
+
+def test_bigvocab_small_batch_gradients():
+    """Every gradient against the oracle at the full width of the big-vocabulary training step
+    (d = 4096, V = 128256, n = 4, r = 16, Zipf targets, balance term on): a batch of 3 positions, which the
+    fp64 oracle finishes in about a minute.  The weight gradients sum over positions and the balance term's
+    gradient depends on the batch's mean gate weights, so they need a batch the oracle can run whole."""
+    from paper_2410_17765_b200 import binding
+
+    big = inputs_for("bigvocab_fwd_bwd", "zipf")
+    s = big.shape
+    sub = synth.subsample_positions(big, torch.tensor([0, 1, 2]))
+    ref = cp_head.backward(sub.h, sub.W_head, sub.E, sub.W_g, sub.x, s.n, s.r, aux_coef=1.0)
+    dev = to_dev(sub)
+    saved = binding.Saved.alloc(binding.make_shape(3, s.d, s.V, s.n, s.r))
+    st = torch.zeros(1, dtype=torch.int32, device="cuda")
+    fwd = binding.forward(*dev, aux_coef=1.0, saved=saved, want_counts=True, dev_status=st)
+    g = binding.backward(*dev, saved, aux_coef=1.0, dev_status=st)
+    torch.cuda.synchronize()
+    assert int(st.item()) == 0
+    reff = cp_head.forward(sub.h, sub.W_head, sub.E, sub.W_g, sub.x, s.n, s.r, aux_coef=1.0)
+    assert np.max(np.abs(fwd["logp"].cpu().numpy() - reff.logp)) <= LOGP_TOL
+    assert abs(float(fwd["loss"].item()) - reff.loss) <= LOGP_TOL
+    assert_expert_counts(fwd["counts"].cpu().numpy(), reff.logw)
+    assert rel_l2(g["dh"].float().cpu().numpy(), ref.dh) <= GRAD_TOL
+    assert rel_l2(g["dW_g"].float().cpu().numpy(), ref.dW_g) <= GRAD_TOL
+    # the gate gradient with the balance term really in it: it differs from the plain one
+    plain = cp_head._coefficients(reff, 3, 0.0, None, None)[1]
+    assert np.linalg.norm(ref.dg - plain) > 1e-3 * np.linalg.norm(plain)
+    assert rel_l2_blocked(g["dW_head"], ref.dW_head) <= GRAD_TOL
+    err_dE = rel_l2_blocked(g["dE"].view(64, -1, s.d), ref.dE.reshape(64, -1, s.d))
+    assert err_dE <= GRAD_TOL, err_dE
 
 
 def test_distill_full_size_sampled_kl_and_dh():

@@ -1,6 +1,5 @@
 """Seeded random shapes through every likelihood entry point, against the oracle: ragged N, V, d
 (multiples of 64), all n and several r, uniform and Zipf targets, chunked and unchunked backward."""
-import os
 
 import numpy as np
 import pytest
@@ -8,6 +7,7 @@ import torch
 
 from oracle import cp_head
 from paper_2410_17765_b200 import synth
+from parity_checks import assert_expert_counts
 
 pytestmark = pytest.mark.gpu
 
@@ -47,18 +47,10 @@ def test_random_shape(it):
     dev = [t.cuda() for t in (inp.h, inp.W_head, inp.E, inp.W_g, inp.x)]
     cs = binding.make_shape(shape.N, shape.d, shape.V, n, r)
     st = torch.zeros(1, dtype=torch.int32, device="cuda")
-    old = os.environ.get("CPMTP_BWD_CHUNK_ROWS")
-    try:
-        if chunk:
-            os.environ["CPMTP_BWD_CHUNK_ROWS"] = str(chunk)
+    with binding.knobs(CPMTP_BWD_CHUNK_ROWS=chunk or None):
         saved = binding.Saved.alloc(cs)
-        f = binding.forward(*dev, aux_coef=aux if aux else None, saved=saved, dev_status=st)
+        f = binding.forward(*dev, aux_coef=aux if aux else None, saved=saved, want_counts=True, dev_status=st)
         g = binding.backward(*dev, saved, aux_coef=aux if aux else None, dev_status=st)
-    finally:
-        if old is None:
-            os.environ.pop("CPMTP_BWD_CHUNK_ROWS", None)
-        else:
-            os.environ["CPMTP_BWD_CHUNK_ROWS"] = old
     sc = binding.score_draft(*dev, dev_status=st)
     saved_f = binding.Saved.alloc_full(cs)
     ff = binding.forward_full(dev[0], W_full.cuda(), dev[3], dev[4], saved=saved_f, dev_status=st)
@@ -69,6 +61,8 @@ def test_random_shape(it):
     assert np.abs(sc["logp_joint"].cpu().numpy() - ref.logp).max() <= 2e-3, shape
     assert abs(float(f["loss"].item()) - ref.loss) <= 2e-3, shape
     assert np.abs(ff["logp"].cpu().numpy() - reff.logp).max() <= 2e-3, shape
+    assert_expert_counts(f["counts"].cpu().numpy(), ref.logw)
+    assert_expert_counts(ff["counts"].cpu().numpy(), reff.logw)
     for key, want in (("dh", refg.dh), ("dW_head", refg.dW_head), ("dE", refg.dE), ("dW_g", refg.dW_g)):
         if np.linalg.norm(want) > 0:
             assert rel_l2(g[key].float().cpu().numpy(), want) <= 1e-2, (shape, key)
@@ -113,20 +107,12 @@ def test_random_distill_shape(it):
     cs = binding.make_shape(shape.N, shape.d, shape.V, n, r)
     st = torch.zeros(1, dtype=torch.int32, device="cuda")
     saved, dsaved = binding.Saved.alloc(cs), binding.DistillSaved.alloc(cs)
-    old = os.environ.get("CPMTP_BWD_CHUNK_ROWS")
-    try:
-        if chunk:
-            os.environ["CPMTP_BWD_CHUNK_ROWS"] = str(chunk)
+    with binding.knobs(CPMTP_BWD_CHUNK_ROWS=chunk or None):
         out = binding.distill_forward(*dev, saved, dsaved, beta=beta, gamma=gamma, aux_coef=aux if aux else None,
                                       dev_status=st)
         g = binding.distill_backward(*dev, saved, dsaved, beta=beta, gamma=gamma, aux_coef=aux if aux else None,
                                      dev_status=st)
         torch.cuda.synchronize()
-    finally:
-        if old is None:
-            os.environ.pop("CPMTP_BWD_CHUNK_ROWS", None)
-        else:
-            os.environ["CPMTP_BWD_CHUNK_ROWS"] = old
     assert int(st.item()) == 0, shape
     assert np.abs(out["kl"].cpu().numpy() - ref.kl).max() <= 2e-3, shape
     assert np.abs(out["logp_prefix"].cpu().numpy() - ref.prefix).max() <= 2e-3, shape

@@ -4,22 +4,21 @@ Some users of the library run where they may not allocate device memory at all:
 a serving process that froze its memory pool at start-up, or an extension that is
 handed tensors but no allocator.  For them the library carries a fixed scratch
 array of its own.  This file checks, through the C-ABI, that the variant returns
-what the ordinary entry point returns, twice in a row (the second call starts
-from the scratch contents the first one left behind), and that shapes too large
-for the fixed array are refused rather than overrunning it.
+what the ordinary entry point returns -- the same kernels on the same schedule, so
+bit for bit -- twice in a row (the second call starts from the scratch contents
+the first one left behind), that the device's free memory does not move across a
+call, and that shapes too large for the fixed array are refused rather than
+overrunning it.
 
 Collected last on purpose (file name), so a failure here cannot hide other tests
 from a run that stops at the first failure.
 """
-import numpy as np
 import pytest
 import torch
 
 from paper_2410_17765_b200 import synth
 
 pytestmark = pytest.mark.gpu
-
-LOGP_TOL = 2e-3
 
 
 def test_static_scratch_scoring_matches_workspace_scoring_twice():
@@ -36,17 +35,25 @@ def test_static_scratch_scoring_matches_workspace_scoring_twice():
         pre_out = {"logp_joint": torch.empty(N, dtype=torch.float32, device="cuda"),
                    "logp_prefix": torch.empty((N, shape.n), dtype=torch.float32, device="cuda")}
         status = torch.zeros(1, dtype=torch.int32, device="cuda")
+        if call == 0:
+            # the very first use of the entry point in a process loads its kernels and looks up the
+            # scratch array's address; do that before memory is measured
+            binding.score_draft_static(*dev, dev_status=status, out=pre_out)
         torch.cuda.synchronize()
-        # cumulative count of blocks torch's allocator has handed out: unchanged if nothing was requested
+        # two witnesses that nothing was allocated: the count of blocks torch's allocator has handed out
+        # (torch-side requests) and the device's free memory as the driver reports it (which a cudaMalloc
+        # made inside the library, invisible to torch, would lower)
         before = torch.cuda.memory_stats()["allocation.all.allocated"]
+        free_before, _ = torch.cuda.mem_get_info()
         got = binding.score_draft_static(*dev, dev_status=status, out=pre_out)
         torch.cuda.synchronize()
+        free_after, _ = torch.cuda.mem_get_info()
         assert torch.cuda.memory_stats()["allocation.all.allocated"] == before
+        assert free_after == free_before
         assert int(status.item()) == 0
         for key in ("logp_joint", "logp_prefix"):
-            a, b = got[key].cpu().numpy(), want[key].cpu().numpy()
-            assert np.all(np.isfinite(a))
-            assert np.max(np.abs(a - b)) <= LOGP_TOL, (call, key)
+            assert bool(torch.isfinite(got[key]).all())
+            assert torch.equal(got[key], want[key]), (call, key)
         outputs[call] = got["logp_joint"].clone()
     assert outputs[0].shape[0] == 8 and outputs[1].shape[0] == 3
 
