@@ -24,8 +24,9 @@
  *  - Return value: CPMTP_OK or a negative error code; on a validation error
  *    nothing was enqueued.  `dev_status` (device int32, may be NULL; the caller
  *    zeroes it) is raised by kernels to 1 if a target token was outside [0, V)
- *    (the token is clamped, the run continues) or 2 if an internal bounded wait
- *    expired (results invalid).
+ *    (the token is clamped, the run continues), 2 if an internal bounded wait
+ *    expired (results invalid), or 3 in the checked build when an index check failed
+ *    (see cpmtp_debug_status).
  *  - Limits: d % 64 == 0, 1 <= r <= 32, 1 <= n <= 8, N >= 1, V >= 2,
  *    N*n*r*d < 2^40.
  *  - CUDA graphs: the entry points only enqueue kernels and copies, so they may be recorded by stream
@@ -132,6 +133,15 @@ typedef struct cpmtp_saved {
 } cpmtp_saved;
 
 typedef struct CUstream_st* cpmtp_stream;
+
+/* Checked build only (libcpmtp_debug.so, compiled with -DCPMTP_DEBUG; there is no counterpart in the paper).
+ * In that build every store and gather of the tensor-core kernels' epilogues, and the candidate gather of
+ * draft generation, first compares the elements it is about to touch with the extent of the buffer; an access
+ * that does not fit is skipped and raises status 3, in `dev_status` and in a per-device word that stays
+ * raised until the library is unloaded.  This call synchronizes the current device and returns that word:
+ * 0 = every index check since the library was loaded has passed, 3 = one failed.  The release library
+ * compiles the checks out and returns -1 here. */
+int cpmtp_debug_status(void);
 
 int cpmtp_version(void);   /* major * 100 + minor * 10; 110 added the distillation entry points, 120 CPMTP_FLAG_ACCUM_GRADS */
 const char* cpmtp_status_string(int status);

@@ -14,7 +14,7 @@ from typing import Optional
 
 import torch
 
-from .build import LIB_PATH
+from .build import DEBUG_LIB_PATH, LIB_PATH
 
 OP_FORWARD, OP_BACKWARD, OP_SCORE, OP_SAMPLE, OP_FORWARD_FULL, OP_BACKWARD_FULL = 0, 1, 2, 3, 4, 5
 OP_DISTILL_FORWARD, OP_DISTILL_BACKWARD = 6, 7
@@ -28,7 +28,7 @@ EXPORTS = [
     "cpmtp_score_draft", "cpmtp_host_staging_bytes", "cpmtp_forward_host", "cpmtp_profile_begin",
     "cpmtp_profile_end", "cpmtp_score_draft_static", "cpmtp_sample_draft",
     "cpmtp_forward_full", "cpmtp_backward_full", "cpmtp_verify_draft",
-    "cpmtp_distill_forward", "cpmtp_distill_backward", "cpmtp_reload_knobs",
+    "cpmtp_distill_forward", "cpmtp_distill_backward", "cpmtp_reload_knobs", "cpmtp_debug_status",
 ]
 
 STATIC_SCRATCH_BYTES = 4 << 20
@@ -60,9 +60,13 @@ def load_library() -> ctypes.CDLL:
     global _lib
     if _lib is not None:
         return _lib
-    if not os.path.exists(LIB_PATH):
-        raise RuntimeError(f"{LIB_PATH} not found: build it with `python -m paper_2410_17765_b200.build`")
-    lib = ctypes.CDLL(LIB_PATH)
+    # CPMTP_LIBRARY=debug selects the checked build (index checks in every epilogue), made by
+    # `python -m paper_2410_17765_b200.build --debug`; any other value is taken as a path
+    choice = os.environ.get("CPMTP_LIBRARY", "")
+    path = LIB_PATH if not choice else DEBUG_LIB_PATH if choice == "debug" else choice
+    if not os.path.exists(path):
+        raise RuntimeError(f"{path} not found: build it with `python -m paper_2410_17765_b200.build`")
+    lib = ctypes.CDLL(path)
     vp, sz, i32p, fp = ctypes.c_void_p, ctypes.c_size_t, ctypes.c_void_p, ctypes.c_void_p
     shp = ctypes.POINTER(CShape)
     svp = ctypes.POINTER(CSaved)
@@ -100,11 +104,18 @@ def load_library() -> ctypes.CDLL:
     lib.cpmtp_distill_backward.argtypes = [shp, vp, vp, vp, vp, i32p, vp, svp, dsp, ctypes.c_float, ctypes.c_float,
                                            fp, fp, vp, vp, vp, vp, vp, sz, i32p, vp]
     lib.cpmtp_reload_knobs.restype = ctypes.c_int
+    lib.cpmtp_debug_status.restype = ctypes.c_int
     lib.cpmtp_profile_begin.restype = ctypes.c_int
     lib.cpmtp_profile_end.restype = ctypes.c_int
     lib.cpmtp_profile_end.argtypes = [ctypes.POINTER(ctypes.c_float), ctypes.POINTER(ctypes.c_int32), ctypes.c_int]
     _lib = lib
     return lib
+
+
+def debug_status() -> int:
+    """cpmtp_debug_status: -1 for the release library; for the checked build 0 while every index check has
+    passed and 3 once one has failed (synchronizes the device)."""
+    return int(load_library().cpmtp_debug_status())
 
 
 def reload_knobs() -> None:

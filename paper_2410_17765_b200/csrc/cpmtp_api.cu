@@ -845,6 +845,17 @@ int cpmtp_reload_knobs(void) {
   return CPMTP_OK;
 }
 
+int cpmtp_debug_status(void) {
+#ifdef CPMTP_DEBUG
+  int seen = 0;
+  if (cudaDeviceSynchronize() != cudaSuccess) return CPMTP_ERR_LAUNCH;
+  if (cudaMemcpyFromSymbol(&seen, g_debug_status, sizeof(int)) != cudaSuccess) return CPMTP_ERR_LAUNCH;
+  return seen;
+#else
+  return -1;   // not a checked build
+#endif
+}
+
 int cpmtp_profile_begin(void) {
   for (cudaEvent_t e : g_prof.events) cudaEventDestroy(e);
   g_prof.events.clear();

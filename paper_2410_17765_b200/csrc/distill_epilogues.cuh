@@ -73,7 +73,7 @@ __device__ __forceinline__ void finish_columns(float* pd, const uint16_t* __rest
     float t[P];
 #pragma unroll
     for (int i = 0; i < P; ++i) t[i] = 0.f;
-    if (row_ok && c < V) {
+    if (row_ok && c < V && CPMTP_INDEX_OK(c, vec ? P : 1, V)) {
       if (vec) {
         if constexpr (P == 8) {
           const uint4 u = __ldg(reinterpret_cast<const uint4*>(trow + c));
@@ -152,7 +152,8 @@ struct EpiKl : EpiDefaults {
     st.acc = 0.f;
   }
   __device__ static void unit_end(const Params& p, State& st, int, int split, int row_in_tile, uint8_t*, int) {
-    if (st.valid) p.part[static_cast<size_t>(st.orow) * p.splits + split] = st.acc;
+    const size_t pi = static_cast<size_t>(st.orow) * p.splits + split;
+    if (st.valid && CPMTP_INDEX_OK(pi, 1, static_cast<size_t>(p.groups) * p.r * p.splits)) p.part[pi] = st.acc;
     // teacher statistics: every lane of the group holds those of its own columns; combine over the group
     float m = st.tm2;
 #pragma unroll
@@ -160,9 +161,10 @@ struct EpiKl : EpiDefaults {
     float l = st.tl > 0.f ? st.tl * ptx::ex2_approx(st.tm2 - m) : 0.f;
 #pragma unroll
     for (int o = R >> 1; o > 0; o >>= 1) l += __shfl_xor_sync(0xffffffffu, l, o);
-    if (st.grp_ok && row_in_tile % R == 0) {
-      p.part_tm[static_cast<size_t>(st.grp) * p.splits + split] = m;
-      p.part_tl[static_cast<size_t>(st.grp) * p.splits + split] = l;
+    const size_t ti = static_cast<size_t>(st.grp) * p.splits + split;
+    if (st.grp_ok && row_in_tile % R == 0 && CPMTP_INDEX_OK(ti, 1, static_cast<size_t>(p.groups) * p.splits)) {
+      p.part_tm[ti] = m;
+      p.part_tl[ti] = l;
     }
   }
   __device__ static void tile(const Params& p, State& st, uint32_t tacc, int, int n_tile, int row_in_tile,
@@ -274,7 +276,8 @@ struct EpiDistillGrad : EpiDefaults {
         for (int j = 0; j < 32; ++j)
           if (j == t) v[j] += st.coef;
       }
-      if (st.valid) store_bf16x32(p.G + static_cast<size_t>(st.orow_local) * p.ldg + col0, v);
+      const size_t gi = static_cast<size_t>(st.orow_local) * p.ldg + col0;
+      if (st.valid && CPMTP_INDEX_OK(gi, 32, static_cast<size_t>(p.groups) * p.r * p.ldg)) store_bf16x32(p.G + gi, v);
     }
   }
 };

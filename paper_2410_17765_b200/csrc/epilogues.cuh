@@ -176,7 +176,8 @@ struct EpiProj : EpiDefaults {
     for (int b = 0; b < BN / 64; ++b) {
       const int col0 = n_tile * BN + b * 64;
       if (col0 >= p.ncols) continue;
-      int tok = __ldg(p.x + static_cast<size_t>(row) * p.n + (col0 / p.d) / p.r);
+      const size_t xi = static_cast<size_t>(row) * p.n + (col0 / p.d) / p.r;
+      int tok = CPMTP_INDEX_OK(xi, 1, static_cast<size_t>(p.M) * p.n) ? __ldg(p.x + xi) : 0;
       if (tok < 0 || tok >= p.V) {
         if (p.dev_status != nullptr) atomicMax(p.dev_status, kDevTargetOutOfRange);
         tok = tok < 0 ? 0 : p.V - 1;
@@ -202,9 +203,11 @@ struct EpiProj : EpiDefaults {
 #pragma unroll
       for (int b = 0; b < BN / 64; ++b)
         if (b == (c >> 6)) tok = st.tok[b];
-      const uint4* src = reinterpret_cast<const uint4*>(p.E + static_cast<size_t>(tok) * p.d + j0);
+      const size_t ei = static_cast<size_t>(tok) * p.d + j0;
+      const uint4* src = reinterpret_cast<const uint4*>(p.E + ei);
+      const bool ok = CPMTP_INDEX_OK(ei, 32, static_cast<size_t>(p.V) * p.d);
 #pragma unroll
-      for (int q = 0; q < 4; ++q) e[q] = __ldg(src + q);
+      for (int q = 0; q < 4; ++q) e[q] = ok ? __ldg(src + q) : make_uint4(0u, 0u, 0u, 0u);
     };
     float part = 0.f;
     auto work = [&](int c, float (&v)[32], const uint4 (&e)[4]) {
@@ -213,7 +216,8 @@ struct EpiProj : EpiDefaults {
       SlabStore::put(smem, epi_tid, v, (c >> 5) & 1);
       if (c & 32) SlabStore::flush(&p.z_map, smem, epi_tid, col0 - 32, m_tile * kBM + (row_in_tile & ~31));
       if (!valid) return;
-      if (p.z32 != nullptr) {
+      if (p.z32 != nullptr &&
+          CPMTP_INDEX_OK(static_cast<size_t>(row) * p.ncols + col0, 32, static_cast<size_t>(p.M) * p.ncols)) {
         float4* dst = reinterpret_cast<float4*>(p.z32 + static_cast<size_t>(row) * p.ncols + col0);
 #pragma unroll
         for (int q = 0; q < 8; ++q) dst[q] = make_float4(v[q * 4], v[q * 4 + 1], v[q * 4 + 2], v[q * 4 + 3]);
@@ -225,7 +229,8 @@ struct EpiProj : EpiDefaults {
       if ((c & 32) == 0) {
         part = acc;
       } else {
-        p.tgt_part[static_cast<size_t>(row) * (p.ncols >> 6) + (col0 >> 6)] = part + acc;
+        const size_t ti = static_cast<size_t>(row) * (p.ncols >> 6) + (col0 >> 6);
+        if (CPMTP_INDEX_OK(ti, 1, static_cast<size_t>(p.M) * (p.ncols >> 6))) p.tgt_part[ti] = part + acc;
       }
     };
     float va[32], vb[32];
@@ -289,9 +294,10 @@ struct EpiLse : EpiDefaults {
   __device__ static void unit_end(const Params& p, State& st, int m_tile, int part, int row_in_tile,
                                   uint8_t*, int) {
     const int row = m_tile * kBM + row_in_tile;
-    if (row < p.M) {
-      p.part_m[static_cast<size_t>(row) * p.parts + part] = st.m2;
-      p.part_l[static_cast<size_t>(row) * p.parts + part] = st.l;
+    const size_t pi = static_cast<size_t>(row) * p.parts + part;
+    if (row < p.M && CPMTP_INDEX_OK(pi, 1, static_cast<size_t>(p.M) * p.parts)) {
+      p.part_m[pi] = st.m2;
+      p.part_l[pi] = st.l;
     }
   }
   __device__ static void tile(const Params& p, State& st, uint32_t tacc, int m_tile, int n_tile,
@@ -301,7 +307,8 @@ struct EpiLse : EpiDefaults {
     for_each_chunk(tacc, 0, chunk_end(tile_col0, BN, p.V), [&](int c, float (&v)[32]) {
       const int col0 = tile_col0 + c;
       if constexpr (STORE) {
-        if (row < p.M) {
+        if (row < p.M &&
+            CPMTP_INDEX_OK(static_cast<size_t>(row) * p.lds + col0, 32, static_cast<size_t>(p.M) * p.lds)) {
           float4* dst = reinterpret_cast<float4*>(p.S + static_cast<size_t>(row) * p.lds + col0);
 #pragma unroll
           for (int q = 0; q < 8; ++q) dst[q] = make_float4(v[q * 4], v[q * 4 + 1], v[q * 4 + 2], v[q * 4 + 3]);
@@ -342,10 +349,12 @@ struct EpiLseFull : EpiDefaults {
   }
   __device__ static void unit_end(const Params& p, State& st, int m_tile, int part, int row_in_tile, uint8_t*, int) {
     const int row = m_tile * kBM + row_in_tile;
-    if (row < p.M && st.k >= 0) {
-      p.part_m[static_cast<size_t>(row) * p.parts + part] = st.m2;
-      p.part_l[static_cast<size_t>(row) * p.parts + part] = st.l;
-      if (st.tok == -2) p.tgt[static_cast<size_t>(row) * p.K + st.k] = st.tgt;   // these columns held the target
+    const size_t pi = static_cast<size_t>(row) * p.parts + part;
+    if (row < p.M && st.k >= 0 && CPMTP_INDEX_OK(pi, 1, static_cast<size_t>(p.M) * p.parts)) {
+      p.part_m[pi] = st.m2;
+      p.part_l[pi] = st.l;
+      const size_t ti = static_cast<size_t>(row) * p.K + st.k;
+      if (st.tok == -2 && CPMTP_INDEX_OK(ti, 1, static_cast<size_t>(p.M) * p.K)) p.tgt[ti] = st.tgt;   // these columns held the target
     }
   }
   __device__ static void tile(const Params& p, State& st, uint32_t tacc, int m_tile, int n_tile, int row_in_tile,
@@ -356,7 +365,8 @@ struct EpiLseFull : EpiDefaults {
     if (st.k != k) {   // first tile of the unit (units never straddle heads)
       st.k = k;
       if (row < p.M) {
-        int tok = p.x[static_cast<size_t>(row) * p.n + k / p.r];
+        const size_t xi = static_cast<size_t>(row) * p.n + k / p.r;
+        int tok = CPMTP_INDEX_OK(xi, 1, static_cast<size_t>(p.M) * p.n) ? p.x[xi] : 0;
         if (tok < 0 || tok >= p.V) {
           if (p.dev_status != nullptr) atomicMax(p.dev_status, kDevTargetOutOfRange);
           tok = tok < 0 ? 0 : p.V - 1;
@@ -431,7 +441,8 @@ struct EpiLogitGrad : EpiDefaults {
       const int k = static_cast<int>(grow - i * p.K);
       st.lse2 = p.lse[grow] * kLog2e;
       st.coef = p.coef[grow];
-      const int tok = p.x[i * p.n + k / p.r];
+      const long long xi = i * p.n + k / p.r;
+      const int tok = CPMTP_INDEX_OK(xi, 1, (p.row0 + p.rows + p.K - 1) / p.K * p.n) ? p.x[xi] : 0;
       st.tok = tok < 0 ? 0 : (tok >= p.V ? p.V - 1 : tok);
     }
   }
@@ -483,7 +494,8 @@ struct EpiLogitGradFull : EpiDefaults {
       if (valid) {
         st.lse2 = p.lse[static_cast<size_t>(row) * p.K + k] * kLog2e;
         st.coef = p.coef[static_cast<size_t>(row) * p.K + k];
-        const int tok = p.x[static_cast<size_t>(row) * p.n + k / p.r];
+        const size_t xi = static_cast<size_t>(row) * p.n + k / p.r;
+        const int tok = CPMTP_INDEX_OK(xi, 1, static_cast<size_t>(p.M) * p.n) ? p.x[xi] : 0;
         st.tok = tok < 0 ? 0 : (tok >= p.V ? p.V - 1 : tok);
       }
     }
@@ -536,13 +548,16 @@ struct EpiStoreBf16 : EpiDefaults {
       const int col0 = tile_col0 + c;
       if constexpr (GATE) {
         for (int b = 0; b < p.r; ++b) {
+          if (!CPMTP_INDEX_OK(static_cast<size_t>(b) * p.ncols + col0, 32, static_cast<size_t>(p.r) * p.ncols)) continue;
           const float g = p.dg[static_cast<size_t>(row) * p.r + b];
           const uint4* w = reinterpret_cast<const uint4*>(p.W_g + static_cast<size_t>(b) * p.ncols + col0);
 #pragma unroll
           for (int q = 0; q < 4; ++q) axpy8(g, __ldg(w + q), v + q * 8);
         }
       }
-      uint16_t* dst = p.C + static_cast<size_t>(row) * p.ldc + col0;
+      const size_t ci = static_cast<size_t>(row) * p.ldc + col0;
+      if (!CPMTP_INDEX_OK(ci, 32, static_cast<size_t>(p.M - 1) * p.ldc + p.ncols)) return;
+      uint16_t* dst = p.C + ci;
       if (p.accumulate) add_bf16x32(dst, v);
       store_bf16x32(dst, v);
     });
@@ -567,7 +582,9 @@ struct EpiAccumF32 : EpiDefaults {
     const int tile_col0 = n_tile * BN;
     for_each_chunk(tacc, 0, chunk_end(tile_col0, BN, p.ncols), [&](int c, float (&v)[32]) {
       if (!valid) return;
-      float4* dst = reinterpret_cast<float4*>(p.C + static_cast<size_t>(row) * p.ldc + tile_col0 + c);
+      const size_t ci = static_cast<size_t>(row) * p.ldc + tile_col0 + c;
+      if (!CPMTP_INDEX_OK(ci, 32, static_cast<size_t>(p.M - 1) * p.ldc + p.ncols)) return;
+      float4* dst = reinterpret_cast<float4*>(p.C + ci);
 #pragma unroll
       for (int q = 0; q < 8; ++q) {
         float4 o = make_float4(v[q * 4 + 0], v[q * 4 + 1], v[q * 4 + 2], v[q * 4 + 3]);

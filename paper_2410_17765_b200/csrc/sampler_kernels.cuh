@@ -15,6 +15,7 @@
 
 #include "../../include/cpmtp.h"
 #include "small_kernels.cuh"
+#include "tc_gemm.cuh"
 
 namespace cpmtp {
 
@@ -294,7 +295,9 @@ draft_step_kernel(const float* __restrict__ S, int lds, const float* __restrict_
       const bool active = job < jobs;
       const int jj = active ? job : 0;
       const int j = jj / r, a = jj - j * r;
-      const uint4* erow = reinterpret_cast<const uint4*>(E + static_cast<size_t>(cand_tok[j]) * d);
+      // a candidate outside the vocabulary would gather from beyond E (checked build: reported, row 0 read instead)
+      const int tok_j = CPMTP_INDEX_OK(cand_tok[j], 1, V) ? cand_tok[j] : 0;
+      const uint4* erow = reinterpret_cast<const uint4*>(E + static_cast<size_t>(tok_j) * d);
       const float4* zrow =
           reinterpret_cast<const float4*>(z32 + (static_cast<size_t>(i) * K + static_cast<size_t>(s) * r + a) * d);
       float acc = dot_e_z(erow, zrow, l16, d >> 3, 16);
@@ -318,6 +321,10 @@ draft_step_kernel(const float* __restrict__ S, int lds, const float* __restrict_
   if (threadIdx.x == 0) {
     draft[static_cast<size_t>(i) * n + s] = cand_tok[topk];
     done[i] = 0u;   // ready for the next step (launches on the stream are ordered)
+#ifdef CPMTP_DEBUG
+    const int seen = *const_cast<volatile int*>(&g_debug_status);
+    if (seen != 0 && dev_status != nullptr) atomicMax(dev_status, seen);
+#endif
   }
   if (threadIdx.x < 32) {
     const int a = threadIdx.x;

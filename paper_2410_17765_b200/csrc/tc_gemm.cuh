@@ -40,6 +40,27 @@ constexpr int kEpiThreads = 128;   // epilogue threads per 128-row block
 constexpr int kDevOk = 0;
 constexpr int kDevTargetOutOfRange = 1;
 constexpr int kDevWaitTimeout = 2;
+constexpr int kDevIndexOutOfRange = 3;   // checked build only, see CPMTP_INDEX_OK
+
+// Checked build (-DCPMTP_DEBUG, libcpmtp_debug.so): every store and every gather of an epilogue first
+// compares the element range it is about to touch with the extent of the buffer it addresses.  A range
+// that does not fit raises status 3 (in a per-device word that cpmtp_debug_status() reads, and from there
+// in the caller's dev_status at the end of the kernel) and the access is skipped; nothing traps.  In the
+// release build the macro is the constant `true` and its arguments are not evaluated.
+#ifdef CPMTP_DEBUG
+__device__ int g_debug_status = 0;
+__device__ __forceinline__ bool index_ok(unsigned long long first, unsigned long long count,
+                                         unsigned long long extent) {
+  if (first + count <= extent && first + count >= first) return true;
+  atomicMax(&g_debug_status, kDevIndexOutOfRange);
+  return false;
+}
+#define CPMTP_INDEX_OK(first, count, extent)                                            \
+  ::cpmtp::index_ok(static_cast<unsigned long long>(first), static_cast<unsigned long long>(count), \
+                    static_cast<unsigned long long>(extent))
+#else
+#define CPMTP_INDEX_OK(first, count, extent) true
+#endif
 
 struct Sched {
   int m_tiles;    // number of (128 * MB)-row tiles
@@ -336,6 +357,12 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
   ptx::tc_fence_after_sync();
   if (warp == 1) ptx::tmem_dealloc(tmem_base, Cfg::TMEM_COLS);
   if (threadIdx.x == 0 && *abort_flag != 0 && dev_status != nullptr) atomicMax(dev_status, kDevWaitTimeout);
+#ifdef CPMTP_DEBUG
+  if (threadIdx.x == 0 && dev_status != nullptr) {
+    const int seen = *const_cast<volatile int*>(&g_debug_status);
+    if (seen != 0) atomicMax(dev_status, seen);
+  }
+#endif
 }
 
 }  // namespace cpmtp

@@ -26,6 +26,25 @@ def test_exports_every_declared_symbol(lib):
         assert getattr(lib, name) is not None
 
 
+def test_checked_build_exports_the_same_symbols():
+    """The checked build (index checks in every epilogue) is the same library plus the checks."""
+    dbg = ctypes.CDLL(build.build(debug=True))
+    for name in binding.EXPORTS:
+        assert getattr(dbg, name) is not None
+    dbg.cpmtp_debug_status.restype = ctypes.c_int
+    # without a device the status word cannot be read: an error code, never "clean"
+    import torch
+
+    if not torch.cuda.is_available():
+        assert dbg.cpmtp_debug_status() < 0
+
+
+def test_release_build_reports_that_it_has_no_index_checks(lib):
+    if os.environ.get("CPMTP_LIBRARY"):
+        pytest.skip("another library was selected")
+    assert binding.debug_status() == -1
+
+
 def test_version_and_status_strings(lib):
     assert lib.cpmtp_version() >= 100
     assert lib.cpmtp_status_string(0) == b"ok"
