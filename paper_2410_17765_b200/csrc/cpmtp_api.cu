@@ -400,7 +400,7 @@ FullBwdLayout full_bwd_layout(const cpmtp_shape& s) {
 
 struct SampleLayout {
   FwdLayout fwd;
-  size_t logits, z32, lb, part_top, part_best, logp_tmp, done, total;
+  size_t logits, z32, lb, part_top, part_best, logp_tmp, done, cand, total;
   int lds, chunks;
 };
 
@@ -413,11 +413,12 @@ SampleLayout sample_layout(const cpmtp_shape& s, int sms) {
   auto take = [&](size_t bytes) { size_t o = off; off = align_up(off + bytes); return o; };
   L.logits = take(sizeof(float) * static_cast<size_t>(L.fwd.M) * L.lds);
   L.z32 = take(sizeof(float) * static_cast<size_t>(L.fwd.M) * s.d);
-  L.lb = take(sizeof(float) * s.N * s.r);
+  L.lb = take(sizeof(float) * static_cast<size_t>(s.n + 1) * s.N * s.r);   // expert weights before every step and after the last
   L.part_top = take(sizeof(Cand) * static_cast<size_t>(s.N) * L.chunks * kMaxTopk);
   L.part_best = take(sizeof(Cand) * static_cast<size_t>(s.N) * L.chunks);
   L.logp_tmp = take(sizeof(float) * s.N);
   L.done = take(sizeof(unsigned int) * s.N);   // per-position count of finished blocks in a draft step
+  L.cand = take(sizeof(int) * static_cast<size_t>(s.n) * s.N * kMaxTopk);   // candidate tokens of every step
   L.total = off;
   return L;
 }
@@ -992,12 +993,19 @@ int cpmtp_sample_draft(const cpmtp_shape* shape, const void* h, const void* W_he
   CPMTP_TRY(cudaMemcpyAsync(lb, logw, sizeof(float) * s.N * s.r, cudaMemcpyDeviceToDevice, st));   // b = w
   const float inv_temp = uniform != nullptr ? 1.0f / temperature : 1.0f;
   unsigned int* done = reinterpret_cast<unsigned int*>(ws + L.done);
+  int* cand = reinterpret_cast<int*>(ws + L.cand);
   CPMTP_TRY(cudaMemsetAsync(done, 0, sizeof(unsigned int) * s.N, st));
   for (int step = 0; step < s.n; ++step) {
     ProfScope prof(CPMTP_STAGE_DRAFT_STEP, st);
     draft_step_kernel<<<dim3(L.chunks, s.N), kSampleThreads, 0, st>>>(
-        logits, L.lds, z32, static_cast<const uint16_t*>(E), s.d, lse, lb, uniform, inv_temp, step, s.V, s.n, s.r,
-        topk, forced, part_top, part_best, done, dev_status, draft, logp_joint, topk_tokens, topk_logp);
+        logits, L.lds, z32, static_cast<const uint16_t*>(E), s.d, lse, lb, uniform, inv_temp, step, s.N, s.V, s.n, s.r,
+        topk, forced, part_top, part_best, done, cand, dev_status, draft, logp_joint, topk_tokens, topk_logp);
+    CPMTP_TRY(cudaGetLastError());
+  }
+  if (topk_logp != nullptr) {   // the last step's candidates (those of the earlier steps rode on the next step's launch)
+    ProfScope prof(CPMTP_STAGE_DRAFT_STEP, st);
+    draft_tail_kernel<<<dim3(topk, s.N), kSampleThreads, 0, st>>>(z32, static_cast<const uint16_t*>(E), s.d, lse, lb, cand,
+                                                                 s.N, s.V, s.n, s.r, topk, topk_logp);
     CPMTP_TRY(cudaGetLastError());
   }
   return CPMTP_OK;
