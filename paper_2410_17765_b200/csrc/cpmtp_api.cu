@@ -400,7 +400,7 @@ FullBwdLayout full_bwd_layout(const cpmtp_shape& s) {
 
 struct SampleLayout {
   FwdLayout fwd;
-  size_t logits, z32, lb, part_top, part_best, logp_tmp, done, cand, total;
+  size_t logits, z32, lb, lb_exact, part_top, part_best, logp_tmp, done, cand, total;
   int lds, chunks;
 };
 
@@ -413,12 +413,13 @@ SampleLayout sample_layout(const cpmtp_shape& s, int sms) {
   auto take = [&](size_t bytes) { size_t o = off; off = align_up(off + bytes); return o; };
   L.logits = take(sizeof(float) * static_cast<size_t>(L.fwd.M) * L.lds);
   L.z32 = take(sizeof(float) * static_cast<size_t>(L.fwd.M) * s.d);
-  L.lb = take(sizeof(float) * static_cast<size_t>(s.n + 1) * s.N * s.r);   // expert weights before every step and after the last
+  L.lb = take(sizeof(float) * static_cast<size_t>(s.n + 1) * s.N * s.r);   // expert weights before every step and after the last,
+  L.lb_exact = take(sizeof(float) * static_cast<size_t>(s.n + 1) * s.N * s.r);   // as selected on, and exact
   L.part_top = take(sizeof(Cand) * static_cast<size_t>(s.N) * L.chunks * kMaxTopk);
   L.part_best = take(sizeof(Cand) * static_cast<size_t>(s.N) * L.chunks);
   L.logp_tmp = take(sizeof(float) * s.N);
   L.done = take(sizeof(unsigned int) * s.N);   // per-position count of finished blocks in a draft step
-  L.cand = take(sizeof(int) * static_cast<size_t>(s.n) * s.N * kMaxTopk);   // candidate tokens of every step
+  L.cand = take(sizeof(int) * static_cast<size_t>(s.n) * s.N * (kMaxTopk + 1));   // candidate and chosen tokens of every step
   L.total = off;
   return L;
 }
@@ -990,23 +991,26 @@ int cpmtp_sample_draft(const cpmtp_shape* shape, const void* h, const void* W_he
                              static_cast<const uint16_t*>(E), static_cast<const uint16_t*>(W_g), nullptr, logp_tmp,
                              nullptr, nullptr, nullptr, nullptr, ws, L.fwd, dev_status, di->sms, st, logits, L.lds, z32);
   if (rf != CPMTP_OK) return rf;
+  float* lb_exact = reinterpret_cast<float*>(ws + L.lb_exact);
   CPMTP_TRY(cudaMemcpyAsync(lb, logw, sizeof(float) * s.N * s.r, cudaMemcpyDeviceToDevice, st));   // b = w
+  CPMTP_TRY(cudaMemcpyAsync(lb_exact, logw, sizeof(float) * s.N * s.r, cudaMemcpyDeviceToDevice, st));
   const float inv_temp = uniform != nullptr ? 1.0f / temperature : 1.0f;
   unsigned int* done = reinterpret_cast<unsigned int*>(ws + L.done);
   int* cand = reinterpret_cast<int*>(ws + L.cand);
   CPMTP_TRY(cudaMemsetAsync(done, 0, sizeof(unsigned int) * s.N, st));
   for (int step = 0; step < s.n; ++step) {
     ProfScope prof(CPMTP_STAGE_DRAFT_STEP, st);
-    draft_step_kernel<<<dim3(L.chunks, s.N), kSampleThreads, 0, st>>>(
-        logits, L.lds, z32, static_cast<const uint16_t*>(E), s.d, lse, lb, uniform, inv_temp, step, s.N, s.V, s.n, s.r,
-        topk, forced, part_top, part_best, done, cand, dev_status, draft, logp_joint, topk_tokens, topk_logp);
-    CPMTP_TRY(cudaGetLastError());
+    CPMTP_TRY(launch_pdl(draft_step_kernel, dim3(L.chunks, s.N), dim3(kSampleThreads), 0, st, logits, L.lds, z32,
+                         static_cast<const uint16_t*>(E), s.d, lse, lb, lb_exact, uniform, inv_temp, step, s.N, s.V, s.n,
+                         s.r, topk, forced, part_top, part_best, done, cand, dev_status, draft, logp_joint, topk_tokens,
+                         topk_logp));
   }
-  if (topk_logp != nullptr) {   // the last step's candidates (those of the earlier steps rode on the next step's launch)
+  if (topk_logp != nullptr || logp_joint != nullptr) {
+    // the last step's exact values (those of the earlier steps rode on the next step's launch)
     ProfScope prof(CPMTP_STAGE_DRAFT_STEP, st);
-    draft_tail_kernel<<<dim3(topk, s.N), kSampleThreads, 0, st>>>(z32, static_cast<const uint16_t*>(E), s.d, lse, lb, cand,
-                                                                 s.N, s.V, s.n, s.r, topk, topk_logp);
-    CPMTP_TRY(cudaGetLastError());
+    CPMTP_TRY(launch_pdl(draft_tail_kernel, dim3(topk + 1, s.N), dim3(kSampleThreads), 0, st, z32,
+                         static_cast<const uint16_t*>(E), s.d, lse, lb_exact, cand, s.N, s.V, s.n, s.r, topk, topk_logp,
+                         logp_joint));
   }
   return CPMTP_OK;
 }

@@ -9,8 +9,9 @@
 // One streaming kernel per token: every block scans a chunk of the vocabulary for one position
 // and leaves its k best tokens; the block that finishes a position last (a counter in global
 // memory, no waiting anywhere) merges the chunks and folds the chosen token's factors into b.
-// The candidates' reported log-probabilities, which no later step needs, are computed by a few
-// blocks of the next launch.  Ties go to the lowest token id, so results are reproducible.
+// The reported log-probabilities (joint and candidates'), which no later selection needs, are
+// recomputed from the unrounded z by a few blocks of the next launch.  Ties go to the lowest
+// token id, so results are reproducible.
 #pragma once
 #include <cstdint>
 
@@ -26,7 +27,7 @@ constexpr int kSampleWarps = kSampleThreads / 32;
 constexpr int kSamplePerThread = 8;                                // vocabulary entries per thread: two groups of four
 constexpr int kSampleChunk = kSampleThreads * kSamplePerThread;   // vocabulary entries per block
 constexpr int kSampleBlocksPerSm = 4;                              // 64 registers per thread: a whole step is one wave
-static_assert(kSamplePerThread == kMaxTopk, "a thread's sorted entries are its candidate list");
+static_assert(kSamplePerThread == kMaxTopk, "a thread's entries are its candidate list");
 
 struct __align__(8) Cand {
   float score;
@@ -44,7 +45,7 @@ __device__ __forceinline__ bool cand_better(float s1, int i1, float s2, int i2) 
   return s1 > s2 || (s1 == s2 && i1 < i2);
 }
 
-// Sorted (best first) list of at most kMaxTopk candidates kept in registers.
+// List of at most kMaxTopk candidates kept in registers; insert() keeps a list that is in order (best first) in order.
 struct TopList {
   float score[kMaxTopk];
   int idx[kMaxTopk];
@@ -55,20 +56,22 @@ struct TopList {
       idx[j] = kNoToken;
     }
   }
-  // Put all eight entries in order with a 19-comparator sorting network (constant indices only).
-  __device__ void sort() {
-#define CPMTP_CSWAP(a, b)                                          \
-  if (cand_better(score[b], idx[b], score[a], idx[a])) {           \
-    const float ts = score[a]; score[a] = score[b]; score[b] = ts; \
-    const int ti = idx[a]; idx[a] = idx[b]; idx[b] = ti;           \
+  // The lane's best entry (entries need not be in order; among equal scores the lowest id).
+  __device__ Cand best() const {
+    Cand b{score[0], idx[0]};
+#pragma unroll
+    for (int j = 1; j < kMaxTopk; ++j)
+      if (cand_better(score[j], idx[j], b.score, b.idx)) b = Cand{score[j], idx[j]};
+    return b;
   }
-    CPMTP_CSWAP(0, 1) CPMTP_CSWAP(2, 3) CPMTP_CSWAP(4, 5) CPMTP_CSWAP(6, 7)
-    CPMTP_CSWAP(0, 2) CPMTP_CSWAP(1, 3) CPMTP_CSWAP(4, 6) CPMTP_CSWAP(5, 7)
-    CPMTP_CSWAP(1, 2) CPMTP_CSWAP(5, 6)
-    CPMTP_CSWAP(0, 4) CPMTP_CSWAP(1, 5) CPMTP_CSWAP(2, 6) CPMTP_CSWAP(3, 7)
-    CPMTP_CSWAP(2, 4) CPMTP_CSWAP(3, 5)
-    CPMTP_CSWAP(1, 2) CPMTP_CSWAP(3, 4) CPMTP_CSWAP(5, 6)
-#undef CPMTP_CSWAP
+  // Empty the entry that holds token id `i` (ids are unique).
+  __device__ void remove(int i) {
+#pragma unroll
+    for (int j = 0; j < kMaxTopk; ++j)
+      if (idx[j] == i) {
+        score[j] = -INFINITY;
+        idx[j] = kNoToken;
+      }
   }
   __device__ void insert(float s, int i, int k) {
     float last_s = -INFINITY;
@@ -96,17 +99,21 @@ struct TopList {
   }
 };
 
+// Warp-wide best candidate (score desc, index asc), the same in every lane: two hardware warp reductions on
+// integers, the maximum of the scores mapped to unsigned keys of the same order, then the lowest id among
+// the lanes that hold it.  Scores are never NaN.
+__device__ __forceinline__ unsigned int order_key(float x) {
+  const unsigned int b = __float_as_uint(x);
+  return (b & 0x80000000u) ? ~b : (b | 0x80000000u);
+}
+__device__ __forceinline__ float key_value(unsigned int k) {
+  return __uint_as_float((k & 0x80000000u) ? (k & 0x7fffffffu) : ~k);
+}
 __device__ __forceinline__ Cand warp_best(Cand c) {
-#pragma unroll
-  for (int o = 16; o > 0; o >>= 1) {
-    const float os = __shfl_xor_sync(0xffffffffu, c.score, o);
-    const int oi = __shfl_xor_sync(0xffffffffu, c.idx, o);
-    if (cand_better(os, oi, c.score, c.idx)) {
-      c.score = os;
-      c.idx = oi;
-    }
-  }
-  return c;
+  const unsigned int key = order_key(c.score);
+  const unsigned int top = __reduce_max_sync(0xffffffffu, key);
+  const int idx = __reduce_min_sync(0xffffffffu, key == top ? c.idx : kNoToken);
+  return Cand{key_value(top), idx};
 }
 
 // Block-wide best candidate (score desc, index asc); result valid in every thread.
@@ -119,29 +126,28 @@ __device__ __forceinline__ Cand block_best(Cand c, Cand* red /* [kSampleWarps] s
   return warp_best(lane < kSampleWarps ? red[lane] : Cand{-INFINITY, kNoToken});
 }
 
-// The k best entries over the sorted lists of a warp's lanes (token ids are unique, so every round
-// has one winner): lane t < k returns the t-th best, the other lanes an empty candidate.
-__device__ __forceinline__ Cand warp_topk(const TopList& mine, int k) {
+// The k best entries over the lists of a warp's lanes, which it empties as it goes (token ids are unique, so
+// every round has one winner): lane t < k returns the t-th best, the other lanes an empty candidate.
+__device__ __forceinline__ Cand warp_topk(TopList& mine, int k) {
   const int lane = threadIdx.x & 31;
-  int head = 0;
   Cand res{-INFINITY, kNoToken};
+  Cand c = mine.best();
   for (int round = 0; round < k; ++round) {
-    Cand c{-INFINITY, kNoToken};
-#pragma unroll
-    for (int j = 0; j < kMaxTopk; ++j)
-      if (j == head) c = Cand{mine.score[j], mine.idx[j]};
     const Cand w = warp_best(c);
-    if (w.idx == c.idx && c.idx != kNoToken) ++head;
+    if (w.idx == c.idx && c.idx != kNoToken) {   // this lane held the winner: its next best comes up
+      mine.remove(w.idx);
+      c = mine.best();
+    }
     if (lane == round) res = w;
   }
   return res;
 }
 
-// The k best entries over the sorted lists of all threads of the block, written to out[0..k) (shared or
-// global) by warp 0: every warp reduces its lanes' lists to one sorted list, then warp 0 does the same with
-// the warps' lists (lane w holds warp w's).  `stage` is shared scratch of kSampleWarps * kMaxTopk candidates.
-// Ends with a barrier.
-__device__ __forceinline__ void block_topk(const TopList& mine, int k, Cand* out, Cand* stage) {
+// The k best entries over the lists of all threads of the block (emptied on the way), written best first to
+// out[0..k) (shared or global) by warp 0: every warp reduces its lanes' lists to one list, then warp 0 does
+// the same with the warps' lists (lane w holds warp w's).  `stage` is shared scratch of kSampleWarps * kMaxTopk candidates.
+// Ends with a barrier.  Exhaustive: block_topk below falls back on it when many entries tie.
+__device__ __forceinline__ void block_topk_merge(TopList& mine, int k, Cand* out, Cand* stage) {
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const Cand w = warp_topk(mine, k);
   __syncthreads();   // `stage` may still be read from a previous use
@@ -165,50 +171,135 @@ __device__ __forceinline__ void block_topk(const TopList& mine, int k, Cand* out
   __syncthreads();
 }
 
+// Shared scratch of block_topk.
+constexpr int kSelectCap = 64;
+static_assert(kSampleWarps * kMaxTopk == 64, "block_topk reads the warps' maxima as two per lane");
+struct SelectScratch {
+  unsigned int wkeys[kSampleWarps * kMaxTopk];   // every warp's k largest lane maxima (as order keys)
+  unsigned int bound;                            // the k-th largest lane maximum of the block
+  int count;
+  Cand cand[kSelectCap];
+  Cand stage[kSampleWarps * kMaxTopk];           // block_topk_merge
+};
+
+// The k best entries over the lists of all threads of the block, written best first to out[0..k) (shared or
+// global) by warp 0; ends with a barrier.  Instead of merging lists, a bound is found first: the k-th largest of
+// the threads' own maxima.  k different threads hold an entry at least that good, so the k-th best entry of the
+// block is no worse, and every entry not below the bound (usually just the k winners) goes into a small
+// candidate array from which one warp picks the k best by (score desc, id asc).  The order in which candidates
+// arrive does not matter, so the result is reproducible.  More than kSelectCap entries at or above the bound
+// (long runs of equal scores): the exhaustive merge.  Keys of real entries are > 0; 0 stands for "none".
+__device__ __forceinline__ void block_topk(TopList& mine, int k, Cand* out, SelectScratch* sc) {
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  unsigned int key[kMaxTopk];
+  unsigned int cur = 0u;
+#pragma unroll
+  for (int j = 0; j < kMaxTopk; ++j) {
+    key[j] = mine.idx[j] != kNoToken ? order_key(mine.score[j]) : 0u;
+    cur = max(cur, key[j]);
+  }
+  for (int round = 0; round < k; ++round) {   // the warp's k largest thread maxima, one per round
+    const unsigned int top = __reduce_max_sync(0xffffffffu, cur);
+    const unsigned int holders = __ballot_sync(0xffffffffu, cur == top);
+    if (lane == __ffs(holders) - 1) cur = 0u;
+    if (lane == 0) sc->wkeys[warp * kMaxTopk + round] = top;
+  }
+  if (threadIdx.x == 0) sc->count = 0;
+  __syncthreads();
+  if (warp == 0) {   // the k-th largest of all warps' lists: lane holds entries lane and lane + 32 of [warps][kMaxTopk]
+    unsigned int a0 = (lane & (kMaxTopk - 1)) < k ? sc->wkeys[lane] : 0u;
+    unsigned int a1 = (lane & (kMaxTopk - 1)) < k ? sc->wkeys[lane + 32] : 0u;
+    unsigned int top = 0u;
+    for (int round = 0; round < k; ++round) {
+      const unsigned int m = max(a0, a1);
+      top = __reduce_max_sync(0xffffffffu, m);
+      const unsigned int holders = __ballot_sync(0xffffffffu, m == top);
+      if (lane == __ffs(holders) - 1) {
+        if (a0 == top) a0 = 0u; else a1 = 0u;
+      }
+    }
+    if (lane == 0) sc->bound = top;
+  }
+  __syncthreads();
+  const unsigned int bound = sc->bound;
+#pragma unroll
+  for (int j = 0; j < kMaxTopk; ++j)
+    if (key[j] != 0u && key[j] >= bound) {
+      const int pos = atomicAdd(&sc->count, 1);
+      if (pos < kSelectCap) sc->cand[pos] = Cand{mine.score[j], mine.idx[j]};
+    }
+  __syncthreads();
+  const int cnt = sc->count;
+  if (cnt > kSelectCap) {
+    block_topk_merge(mine, k, out, sc->stage);
+    return;
+  }
+  if (warp == 0) {
+    Cand c0 = lane < cnt ? sc->cand[lane] : Cand{-INFINITY, kNoToken};
+    Cand c1 = lane + 32 < cnt ? sc->cand[lane + 32] : Cand{-INFINITY, kNoToken};
+    Cand res{-INFINITY, kNoToken};
+    for (int round = 0; round < k; ++round) {
+      const bool first = cand_better(c0.score, c0.idx, c1.score, c1.idx);
+      const Cand m = first ? c0 : c1;
+      const Cand w = warp_best(m);
+      if (w.idx == m.idx && m.idx != kNoToken) {
+        if (first) c0 = Cand{-INFINITY, kNoToken}; else c1 = Cand{-INFINITY, kNoToken};
+      }
+      if (lane == round) res = w;
+    }
+    if (lane < k) out[lane] = res;
+  }
+  __syncthreads();
+}
+
 // mix[j] = logsumexp_a(S[a, v + j] + off[a]) for the four vocabulary entries v .. v + 3 (16-byte aligned row
-// pieces).  Up to eight experts: all rows are fetched at once and both passes (maximum, sum of exponentials)
-// run from registers; more experts: two passes over memory, the second of which hits the caches.
-__device__ __forceinline__ void mix_of_four(const float* __restrict__ Srow, int lds, int v, int r,
-                                            const float* off_s, float (&mix)[4]) {
+// pieces); off2 = off * log2(e), and the sums run in the log2 domain.  Up to eight experts (`fetched`): the rows
+// were fetched into q by fetch_four and both passes (maximum, sum of exponentials) run from registers; more
+// experts: two passes over memory, the second of which hits the caches.
+__device__ __forceinline__ void fetch_four(const float* __restrict__ Srow, int lds, int v, int r, float4 (&q)[8]) {
+#pragma unroll
+  for (int a = 0; a < 8; ++a)
+    if (a < r) q[a] = __ldg(reinterpret_cast<const float4*>(Srow + static_cast<size_t>(a) * lds + v));
+}
+__device__ __forceinline__ void mix_of_four(const float* __restrict__ Srow, int lds, int v, int r, bool fetched,
+                                            float4 (&q)[8], const float* off2_s, float (&mix)[4]) {
+  constexpr float kL2e = 1.4426950408889634f, kLn2f = 0.6931471805599453f;
   float m[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
   float l[4] = {0.f, 0.f, 0.f, 0.f};
-  if (r <= 8) {
-    float4 q[8];
-#pragma unroll
-    for (int a = 0; a < 8; ++a)
-      if (a < r) q[a] = __ldg(reinterpret_cast<const float4*>(Srow + static_cast<size_t>(a) * lds + v));
+  if (fetched) {
 #pragma unroll
     for (int a = 0; a < 8; ++a)
       if (a < r) {
-        const float off = off_s[a];
-        q[a].x += off; q[a].y += off; q[a].z += off; q[a].w += off;
+        const float off = off2_s[a];
+        q[a].x = fmaf(q[a].x, kL2e, off); q[a].y = fmaf(q[a].y, kL2e, off);
+        q[a].z = fmaf(q[a].z, kL2e, off); q[a].w = fmaf(q[a].w, kL2e, off);
         m[0] = fmaxf(m[0], q[a].x); m[1] = fmaxf(m[1], q[a].y);
         m[2] = fmaxf(m[2], q[a].z); m[3] = fmaxf(m[3], q[a].w);
       }
 #pragma unroll
     for (int a = 0; a < 8; ++a)
       if (a < r) {
-        l[0] += __expf(q[a].x - m[0]); l[1] += __expf(q[a].y - m[1]);
-        l[2] += __expf(q[a].z - m[2]); l[3] += __expf(q[a].w - m[3]);
+        l[0] += ptx::ex2_approx(q[a].x - m[0]); l[1] += ptx::ex2_approx(q[a].y - m[1]);
+        l[2] += ptx::ex2_approx(q[a].z - m[2]); l[3] += ptx::ex2_approx(q[a].w - m[3]);
       }
   } else {
 #pragma unroll 4
     for (int a = 0; a < r; ++a) {
-      const float4 q = __ldg(reinterpret_cast<const float4*>(Srow + static_cast<size_t>(a) * lds + v));
-      const float off = off_s[a];
-      m[0] = fmaxf(m[0], q.x + off); m[1] = fmaxf(m[1], q.y + off);
-      m[2] = fmaxf(m[2], q.z + off); m[3] = fmaxf(m[3], q.w + off);
+      const float4 w = __ldg(reinterpret_cast<const float4*>(Srow + static_cast<size_t>(a) * lds + v));
+      const float off = off2_s[a];
+      m[0] = fmaxf(m[0], fmaf(w.x, kL2e, off)); m[1] = fmaxf(m[1], fmaf(w.y, kL2e, off));
+      m[2] = fmaxf(m[2], fmaf(w.z, kL2e, off)); m[3] = fmaxf(m[3], fmaf(w.w, kL2e, off));
     }
 #pragma unroll 4
     for (int a = 0; a < r; ++a) {
-      const float4 q = __ldg(reinterpret_cast<const float4*>(Srow + static_cast<size_t>(a) * lds + v));
-      const float off = off_s[a];
-      l[0] += __expf(q.x + off - m[0]); l[1] += __expf(q.y + off - m[1]);
-      l[2] += __expf(q.z + off - m[2]); l[3] += __expf(q.w + off - m[3]);
+      const float4 w = __ldg(reinterpret_cast<const float4*>(Srow + static_cast<size_t>(a) * lds + v));
+      const float off = off2_s[a];
+      l[0] += ptx::ex2_approx(fmaf(w.x, kL2e, off) - m[0]); l[1] += ptx::ex2_approx(fmaf(w.y, kL2e, off) - m[1]);
+      l[2] += ptx::ex2_approx(fmaf(w.z, kL2e, off) - m[2]); l[3] += ptx::ex2_approx(fmaf(w.w, kL2e, off) - m[3]);
     }
   }
 #pragma unroll
-  for (int j = 0; j < 4; ++j) mix[j] = m[j] + __logf(l[j]);
+  for (int j = 0; j < 4; ++j) mix[j] = (m[j] + ptx::lg2_approx(l[j])) * kLn2f;
 }
 
 // Exact logits of one token for all r experts of draft step s at position i, from the unrounded z:
@@ -224,19 +315,25 @@ __device__ __forceinline__ void block_token_logits(const uint16_t* __restrict__ 
   for (int a0 = 0; a0 < r; a0 += 4) {
     float acc[4] = {0.f, 0.f, 0.f, 0.f};
     for (int g = threadIdx.x; g < (d >> 3); g += kSampleThreads) {
+      // all nine loads of this piece are issued before the first is used (experts beyond r re-read expert
+      // r - 1 and are dropped below), so the piece costs one round trip to memory, not five
       const uint4 e = __ldg(erow + g);
+      float4 z0[4], z1[4];
+#pragma unroll
+      for (int u = 0; u < 4; ++u) {
+        const int a = min(a0 + u, r - 1);
+        const float4* zrow = reinterpret_cast<const float4*>(z32 + (row0 + a) * d);
+        z0[u] = __ldg(zrow + 2 * g);
+        z1[u] = __ldg(zrow + 2 * g + 1);
+      }
       const float e0 = ptx::bf16_lo(e.x), e1 = ptx::bf16_hi(e.x), e2 = ptx::bf16_lo(e.y), e3 = ptx::bf16_hi(e.y);
       const float e4 = ptx::bf16_lo(e.z), e5 = ptx::bf16_hi(e.z), e6 = ptx::bf16_lo(e.w), e7 = ptx::bf16_hi(e.w);
 #pragma unroll
       for (int u = 0; u < 4; ++u) {
-        if (a0 + u < r) {
-          const float4* zrow = reinterpret_cast<const float4*>(z32 + (row0 + a0 + u) * d);
-          const float4 z0 = __ldg(zrow + 2 * g), z1 = __ldg(zrow + 2 * g + 1);
-          float t = acc[u];
-          t = fmaf(e0, z0.x, t); t = fmaf(e1, z0.y, t); t = fmaf(e2, z0.z, t); t = fmaf(e3, z0.w, t);
-          t = fmaf(e4, z1.x, t); t = fmaf(e5, z1.y, t); t = fmaf(e6, z1.z, t); t = fmaf(e7, z1.w, t);
-          acc[u] = t;
-        }
+        float t = acc[u];
+        t = fmaf(e0, z0[u].x, t); t = fmaf(e1, z0[u].y, t); t = fmaf(e2, z0[u].z, t); t = fmaf(e3, z0[u].w, t);
+        t = fmaf(e4, z1[u].x, t); t = fmaf(e5, z1[u].y, t); t = fmaf(e6, z1[u].z, t); t = fmaf(e7, z1[u].w, t);
+        acc[u] = t;
       }
     }
 #pragma unroll
@@ -255,72 +352,100 @@ __device__ __forceinline__ void block_token_logits(const uint16_t* __restrict__ 
   __syncthreads();
 }
 
-// Conditional log-probabilities of the candidates of draft step s at position i (the reported values, from the
-// unrounded z):  topk_logp[i, s, j] = logsumexp_a(log b_a + log P^(s)(cand_j | a)) - logsumexp_a log b_a,
-// with b the expert weights BEFORE step s.  This block takes candidates j = first, first + stride, ...
-__device__ __forceinline__ void candidate_logps(const uint16_t* __restrict__ E, const float* __restrict__ z32,
-                                                const float* __restrict__ lse, const float* __restrict__ lb_before,
-                                                const int* __restrict__ cand, int i, int s, int d, int V, int n, int r,
-                                                int topk, int first, int stride, float* __restrict__ topk_logp,
-                                                float* tgt_s, float* red) {
+// The reported values of draft step s at position i, from the unrounded z, which no later selection depends on.
+// Job j < topk:  topk_logp[i, s, j] = logsumexp_a(log b_a + log P^(s)(cand_j | a)) - logsumexp_a log b_a, with b the
+// exact expert weights before step s (lb_exact[s]).  Job j == topk: fold the chosen token into the exact weights,
+// lb_exact[s + 1] = lb_exact[s] + log P^(s)(token | .), and after the last step write the joint log-probability.
+// This block takes jobs first, first + stride, ...; tok_hist holds kMaxTopk candidates and then the chosen token.
+__device__ __forceinline__ void exact_step_values(const uint16_t* __restrict__ E, const float* __restrict__ z32,
+                                                  const float* __restrict__ lse, float* __restrict__ lb_exact,
+                                                  const int* __restrict__ tok_hist, int i, int s, int d, int N, int V, int n,
+                                                  int r, int topk, int first, int stride, float* __restrict__ topk_logp,
+                                                  float* __restrict__ logp_joint, float* tgt_s, float* red) {
   const size_t row0 = (static_cast<size_t>(i) * n + s) * r;
-  for (int j = first; j < topk; j += stride) {
-    // a candidate outside the vocabulary would gather from beyond E (checked build: reported, row 0 read instead)
-    int tok = cand[j];
+  const float* lb_before = lb_exact + (static_cast<size_t>(s) * N + i) * r;
+  float* lb_after = lb_exact + (static_cast<size_t>(s + 1) * N + i) * r;
+  const int* toks = tok_hist + (static_cast<size_t>(s) * N + i) * (kMaxTopk + 1);
+  for (int j = first; j <= topk; j += stride) {
+    const bool chosen = j == topk;
+    if (!chosen && topk_logp == nullptr) continue;
+    // a token outside the vocabulary would gather from beyond E (checked build: reported, row 0 read instead)
+    int tok = toks[chosen ? kMaxTopk : j];
     if (!CPMTP_INDEX_OK(tok, 1, V)) tok = 0;
     block_token_logits(E, tok, z32, lse, row0, d, r, tgt_s, red);
     if (threadIdx.x < 32) {
       const int a = threadIdx.x;
-      const float b = a < r ? lb_before[static_cast<size_t>(i) * r + a] : -INFINITY;
-      const float mb = warp_max(b);
-      const float norm = mb + logf(warp_sum(a < r ? expf(b - mb) : 0.f));
+      const float b = a < r ? lb_before[a] : -INFINITY;
       const float x = a < r ? b + tgt_s[a] : -INFINITY;
       const float m = warp_max(x);
-      const float tot = warp_sum(a < r ? expf(x - m) : 0.f);
-      if (a == 0) topk_logp[(static_cast<size_t>(i) * n + s) * topk + j] = m + logf(tot) - norm;
+      const float lp = m + logf(warp_sum(a < r ? expf(x - m) : 0.f));
+      if (chosen) {
+        if (a < r) lb_after[a] = x;
+        if (s == n - 1 && logp_joint != nullptr && a == 0) logp_joint[i] = lp;
+      } else {
+        const float mb = warp_max(b);
+        const float norm = mb + logf(warp_sum(a < r ? expf(b - mb) : 0.f));
+        if (a == 0) topk_logp[(static_cast<size_t>(i) * n + s) * topk + j] = lp - norm;
+      }
     }
-    __syncthreads();   // tgt_s and red are reused by the next candidate
+    __syncthreads();   // tgt_s and red are reused by the next job
   }
 }
 
-// One draft step.  Grid (chunks, N), kSampleThreads threads, lb_hist = [n + 1][N][r] (expert weights before
-// every step), cand_hist = [n][N][kMaxTopk] (candidate tokens of every step).
+// One draft step.  Grid (chunks, N), kSampleThreads threads.
+//   lb_sel   [n + 1][N][r]  expert weights as the SELECTION sees them before every step: the chosen tokens' factors
+//                           are read from the stored logits S (computed from bf16-rounded z, like all of S)
+//   lb_exact [n + 1][N][r]  the same from the unrounded z: what the reported log-probabilities are made of
+//   tok_hist [n][N][kMaxTopk + 1]  candidate tokens of every step, then the chosen one
 //   phase 1 (every block): scan the chunk's entries of position i, mix[v] = logsumexp_a(log b_a + S[s,a,v] - lse[s,a]);
 //            keep the k best tokens and, when sampling, the best Gumbel-perturbed score; write them to part_*.
 //   phase 2 (the block that raises done[i] to the chunk count, i.e. the last to finish for position i): merge the
-//            chunks, choose the token, recompute the chosen token's logits from the unrounded z (fp32; only the
-//            *selection* sees bf16-rounded z), fold them into log b for the next step, and reset done[i].
-//   side job (blocks with chunk < topk, after their own part): the exact conditional log-probabilities of the
-//            candidates of the PREVIOUS step, which nothing later depends on; draft_tail_kernel does the same for
+//            chunks, choose the token, fold its stored logits into lb_sel for the next step, and reset done[i].
+//   side jobs (blocks with chunk <= topk, after their own part): the exact values of the PREVIOUS step (see
+//            exact_step_values), which nothing on the selection path waits for; draft_tail_kernel does the same for
 //            the last step.
 // No block waits for another: whichever finishes last does the merge.
 __global__ void __launch_bounds__(kSampleThreads, kSampleBlocksPerSm)
 draft_step_kernel(const float* __restrict__ S, int lds, const float* __restrict__ z32, const uint16_t* __restrict__ E,
-                  int d, const float* __restrict__ lse, float* __restrict__ lb_hist, const float* __restrict__ uniform,
-                  float inv_temp, int s, int N, int V, int n, int r, int topk, const int32_t* __restrict__ forced,
-                  Cand* __restrict__ part_top, Cand* __restrict__ part_best, unsigned int* __restrict__ done,
-                  int* __restrict__ cand_hist, int* __restrict__ dev_status, int32_t* __restrict__ draft,
-                  float* __restrict__ logp_joint, int32_t* __restrict__ topk_tokens, float* __restrict__ topk_logp) {
+                  int d, const float* __restrict__ lse, float* __restrict__ lb_sel, float* __restrict__ lb_exact,
+                  const float* __restrict__ uniform, float inv_temp, int s, int N, int V, int n, int r, int topk,
+                  const int32_t* __restrict__ forced, Cand* __restrict__ part_top, Cand* __restrict__ part_best,
+                  unsigned int* __restrict__ done, int* __restrict__ tok_hist, int* __restrict__ dev_status,
+                  int32_t* __restrict__ draft, float* __restrict__ logp_joint, int32_t* __restrict__ topk_tokens,
+                  float* __restrict__ topk_logp) {
   __shared__ float off_s[CPMTP_MAX_R];
   __shared__ float lb_s[CPMTP_MAX_R];
   __shared__ float tgt_s[CPMTP_MAX_R];                  // log P^(s)(token | expert)
   __shared__ float red_f[kSampleWarps * CPMTP_MAX_R];
   __shared__ float norm_s;
   __shared__ Cand red[kSampleWarps];
-  __shared__ Cand stage[kSampleWarps * kMaxTopk];
+  __shared__ SelectScratch select;
   __shared__ Cand final_top[kMaxTopk];
   __shared__ int tok_s;
   __shared__ bool is_last;
   const int chunk = blockIdx.x, chunks = gridDim.x, i = blockIdx.y;
   const int K = n * r;
-  const float* lb = lb_hist + static_cast<size_t>(s) * N * r;              // before this step
-  float* lb_next = lb_hist + static_cast<size_t>(s + 1) * N * r;           // after it
+  // Launched with programmatic stream serialization: the next step's blocks may become resident while this
+  // step's last blocks still merge.  What they do before grid_dep_wait() touches only the stored logits, which
+  // no draft step writes: the first half of the scan's loads is in flight while the step before finishes.
+  ptx::grid_dep_launch();
+  const float* Srow = S + (static_cast<size_t>(i) * K + static_cast<size_t>(s) * r) * lds;
+  const int v_end = min(V, (chunk + 1) * kSampleChunk);
+  const bool fetched = r <= 8;
+  float4 q[8];
+  {
+    const int v0 = chunk * kSampleChunk + 4 * threadIdx.x;
+    if (fetched && v0 < v_end) fetch_four(Srow, lds, v0, r, q);
+  }
+  ptx::grid_dep_wait();
+  const float* lb = lb_sel + static_cast<size_t>(s) * N * r;              // before this step
+  float* lb_next = lb_sel + static_cast<size_t>(s + 1) * N * r;           // after it
   if (threadIdx.x < 32) {
     const int a = threadIdx.x;
     const float b = a < r ? lb[static_cast<size_t>(i) * r + a] : -INFINITY;
     if (a < r) {
       lb_s[a] = b;
-      off_s[a] = b - lse[static_cast<size_t>(i) * K + s * r + a];
+      off_s[a] = (b - lse[static_cast<size_t>(i) * K + s * r + a]) * 1.4426950408889634f;   // log2 domain
     }
     const float m = warp_max(b);
     const float e = a < r ? expf(b - m) : 0.f;
@@ -331,12 +456,10 @@ draft_step_kernel(const float* __restrict__ S, int lds, const float* __restrict_
   const float norm = norm_s;
   // ---- phase 1: this block's chunk
   {
-    const float* Srow = S + (static_cast<size_t>(i) * K + static_cast<size_t>(s) * r) * lds;
     const float* urow = uniform != nullptr ? uniform + (static_cast<size_t>(i) * n + s) * V : nullptr;
     TopList top;
     top.init();
     Cand best{-INFINITY, kNoToken};
-    const int v_end = min(V, (chunk + 1) * kSampleChunk);
     // two groups of four consecutive vocabulary entries per thread, half a chunk apart (lds % 32 == 0: 16-byte
     // aligned loads, a warp reads 512 contiguous bytes of every row; entries in [V, lds) exist in the buffer
     // and are left out below)
@@ -345,7 +468,8 @@ draft_step_kernel(const float* __restrict__ S, int lds, const float* __restrict_
       const int v0 = chunk * kSampleChunk + grp * (kSampleChunk / 2) + 4 * threadIdx.x;
       if (v0 >= v_end) continue;
       float mix[4];
-      mix_of_four(Srow, lds, v0, r, off_s, mix);
+      if (grp == 1 && fetched) fetch_four(Srow, lds, v0, r, q);   // (the first group's rows were fetched above)
+      mix_of_four(Srow, lds, v0, r, fetched, q, off_s, mix);
 #pragma unroll
       for (int j = 0; j < 4; ++j) {
         const int v = v0 + j;
@@ -357,8 +481,7 @@ draft_step_kernel(const float* __restrict__ S, int lds, const float* __restrict_
         if (cand_better(sc, v, best.score, best.idx)) best = Cand{sc, v};
       }
     }
-    top.sort();
-    block_topk(top, topk, part_top + (static_cast<size_t>(i) * chunks + chunk) * kMaxTopk, stage);
+    block_topk(top, topk, part_top + (static_cast<size_t>(i) * chunks + chunk) * kMaxTopk, &select);
     if (urow != nullptr) {
       const Cand b = block_best(best, red);
       if (threadIdx.x == 0) part_best[static_cast<size_t>(i) * chunks + chunk] = b;
@@ -374,22 +497,32 @@ draft_step_kernel(const float* __restrict__ S, int lds, const float* __restrict_
   __syncthreads();
   if (is_last) {
     __threadfence();   // the other blocks' partial results, published before their increments, are read below
-    // ---- phase 2: merge (thread t holds the sorted lists of chunks t, t + 256, ...), choose, fold
+    // ---- phase 2: merge (thread t holds the lists of chunks t, t + 256, ..., each written best first), choose, fold
     TopList top;
     top.init();
     Cand best{-INFINITY, kNoToken};
     for (int c = threadIdx.x; c < chunks; c += kSampleThreads) {
       const Cand* src = part_top + (static_cast<size_t>(i) * chunks + c) * kMaxTopk;
-      for (int j = 0; j < topk; ++j) {
-        const Cand pt = load_cand_cg(src + j);
-        if (pt.idx != kNoToken) top.insert(pt.score, pt.idx, topk);
+      Cand got[kMaxTopk];
+#pragma unroll
+      for (int j = 0; j < kMaxTopk; ++j) got[j] = j < topk ? load_cand_cg(src + j) : Cand{-INFINITY, kNoToken};
+      if (c == static_cast<int>(threadIdx.x)) {   // the thread's first list is taken as it is
+#pragma unroll
+        for (int j = 0; j < kMaxTopk; ++j) {
+          top.score[j] = got[j].score;
+          top.idx[j] = got[j].idx;
+        }
+      } else {
+#pragma unroll
+        for (int j = 0; j < kMaxTopk; ++j)
+          if (got[j].idx != kNoToken) top.insert(got[j].score, got[j].idx, topk);
       }
       if (uniform != nullptr) {
         const Cand pb = load_cand_cg(part_best + static_cast<size_t>(i) * chunks + c);
         if (cand_better(pb.score, pb.idx, best.score, best.idx)) best = pb;
       }
     }
-    block_topk(top, topk, final_top, stage);
+    block_topk(top, topk, final_top, &select);
     if (uniform != nullptr) best = block_best(best, red);
     if (threadIdx.x == 0) {   // the drafted token: the caller's, if one is given for this step
       int tok = uniform != nullptr ? best.idx : final_top[0].idx;
@@ -405,36 +538,25 @@ draft_step_kernel(const float* __restrict__ S, int lds, const float* __restrict_
       if (!CPMTP_INDEX_OK(tok, 1, V)) tok = 0;
       tok_s = tok;
       draft[static_cast<size_t>(i) * n + s] = tok;
+      tok_hist[(static_cast<size_t>(s) * N + i) * (kMaxTopk + 1) + kMaxTopk] = tok;
       done[i] = 0u;   // ready for the next step (launches on the stream are ordered)
     }
     if (threadIdx.x < topk) {
       const int t = final_top[threadIdx.x].idx;
-      cand_hist[(static_cast<size_t>(s) * N + i) * kMaxTopk + threadIdx.x] = t;
+      tok_hist[(static_cast<size_t>(s) * N + i) * (kMaxTopk + 1) + threadIdx.x] = t;
       if (topk_tokens != nullptr) topk_tokens[(static_cast<size_t>(i) * n + s) * topk + threadIdx.x] = t;
     }
     __syncthreads();
-    block_token_logits(E, tok_s, z32, lse, (static_cast<size_t>(i) * n + s) * r, d, r, tgt_s, red_f);
-    if (threadIdx.x < 32) {
-      const int a = threadIdx.x;
-      float bb = -INFINITY;
-      if (a < r) {
-        bb = lb_s[a] + tgt_s[a];
-        lb_next[static_cast<size_t>(i) * r + a] = bb;
-      }
-      if (s == n - 1 && logp_joint != nullptr) {
-        const float m = warp_max(bb);
-        const float e = a < r ? expf(bb - m) : 0.f;
-        const float tot = warp_sum(e);
-        if (a == 0) logp_joint[i] = m + logf(tot);
-      }
-    }
-    __syncthreads();
+    if (threadIdx.x < r)   // the chosen token's factors as the selection sees them: its stored logits
+      lb_next[static_cast<size_t>(i) * r + threadIdx.x] =
+          lb_s[threadIdx.x] + __ldg(Srow + static_cast<size_t>(threadIdx.x) * lds + tok_s) -
+          lse[static_cast<size_t>(i) * K + s * r + threadIdx.x];
   }
-  // ---- side job: reported log-probabilities of the previous step's candidates
-  if (s > 0 && topk_logp != nullptr && chunk < topk) {
-    candidate_logps(E, z32, lse, lb_hist + static_cast<size_t>(s - 1) * N * r,
-                    cand_hist + (static_cast<size_t>(s - 1) * N + i) * kMaxTopk, i, s - 1, d, V, n, r, topk, chunk,
-                    chunks, topk_logp, tgt_s, red_f);
+  // ---- side jobs: the exact values of the previous step
+  if (s > 0 && chunk <= topk && (topk_logp != nullptr || logp_joint != nullptr)) {
+    __syncthreads();
+    exact_step_values(E, z32, lse, lb_exact, tok_hist, i, s - 1, d, N, V, n, r, topk, chunk, chunks, topk_logp, logp_joint,
+                      tgt_s, red_f);
   }
 #ifdef CPMTP_DEBUG
   if (threadIdx.x == 0 && dev_status != nullptr) {
@@ -444,17 +566,16 @@ draft_step_kernel(const float* __restrict__ S, int lds, const float* __restrict_
 #endif
 }
 
-// The candidates' reported log-probabilities for the last draft step.  Grid (topk, N).
+// The exact values of the last draft step.  Grid (min(topk + 1, anything >= 1), N).
 __global__ void __launch_bounds__(kSampleThreads, kSampleBlocksPerSm)
 draft_tail_kernel(const float* __restrict__ z32, const uint16_t* __restrict__ E, int d, const float* __restrict__ lse,
-                  const float* __restrict__ lb_hist, const int* __restrict__ cand_hist, int N, int V, int n, int r,
-                  int topk, float* __restrict__ topk_logp) {
+                  float* __restrict__ lb_exact, const int* __restrict__ tok_hist, int N, int V, int n, int r, int topk,
+                  float* __restrict__ topk_logp, float* __restrict__ logp_joint) {
   __shared__ float tgt_s[CPMTP_MAX_R];
   __shared__ float red_f[kSampleWarps * CPMTP_MAX_R];
-  const int i = blockIdx.y, s = n - 1;
-  candidate_logps(E, z32, lse, lb_hist + static_cast<size_t>(s) * N * r,
-                  cand_hist + (static_cast<size_t>(s) * N + i) * kMaxTopk, i, s, d, V, n, r, topk, blockIdx.x, gridDim.x,
-                  topk_logp, tgt_s, red_f);
+  ptx::grid_dep_wait();   // the last step's tokens come from the launch before this one
+  exact_step_values(E, z32, lse, lb_exact, tok_hist, blockIdx.y, n - 1, d, N, V, n, r, topk, blockIdx.x, gridDim.x,
+                    topk_logp, logp_joint, tgt_s, red_f);
 }
 
 // Draft verification: one thread per position.

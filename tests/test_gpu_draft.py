@@ -109,6 +109,32 @@ def test_draft_is_deterministic_and_validates_arguments():
         binding.sample_draft(*dev, shape.n, uniform=torch.rand((4, 2, 900), device="cuda"), temperature=0.0)
 
 
+def test_long_runs_of_equal_scores_go_to_the_lowest_ids():
+    """Whole stretches of the vocabulary with exactly equal scores (here: identical rows of E, so identical logits
+    for every expert) are more ties than the candidate array of the selection holds, so the exhaustive merge runs;
+    the result is still the oracle's: ties resolve to the lowest token id."""
+    from paper_2410_17765_b200 import binding
+
+    shape = synth.Shape(N=3, d=128, V=5000, n=2, r=4)
+    inp = synth.make_inputs(shape, seed=3, weight_scale=2.0)
+    E = inp.E.clone()
+    E[:] = E[0]                       # every token the same: all scores equal
+    E[4000:4003] = inp.E[1] * 4       # three tokens that stand out, inside a later chunk
+    ref = cp_head.draft(inp.h, inp.W_head, E, inp.W_g, shape.n, shape.r, topk=8)
+    st = torch.zeros(1, dtype=torch.int32, device="cuda")
+    out = binding.sample_draft(inp.h.cuda(), inp.W_head.cuda(), E.cuda(), inp.W_g.cuda(), shape.n, topk=8, dev_status=st)
+    torch.cuda.synchronize()
+    assert int(st.item()) == 0
+    tk = out["topk_tokens"].cpu().numpy()
+    # the equal-score tokens that fill the remaining places are the lowest ids, in order
+    for i in range(shape.N):
+        for t in range(shape.n):
+            rest = [v for v in tk[i, t].tolist() if not 4000 <= v < 4003]
+            assert rest == list(range(len(rest))), (i, t, tk[i, t])
+            assert set(tk[i, t].tolist()) == set(ref.topk_tokens[i, t].tolist())
+    assert np.max(np.abs(np.sort(out["topk_logp"].cpu().numpy(), axis=2) - np.sort(ref.topk_logp, axis=2))) <= LOGP_TOL
+
+
 def test_verify_draft_matches_oracle():
     from paper_2410_17765_b200 import binding
 
