@@ -226,6 +226,11 @@ int cpmtp_score_draft(const cpmtp_shape* shape, const void* h, const void* W_hea
  *   topk_tokens [N,n,topk] int32 / topk_logp [N,n,topk] fp32 out or NULL: the
  *     candidates, best first, with their conditional log-probabilities (for a
  *     static draft tree as in the speculative-decoding section).
+ * Precision: the SELECTION of a token (and of the candidate set) works on logits computed from the
+ * bf16-rounded projected hidden state, both for the step's own factors and for the factors of the tokens
+ * already drawn, so among tokens whose probabilities differ by less than about 1 % the choice may differ from
+ * exact arithmetic; every VALUE returned (logp_joint, topk_logp) is recomputed from the unrounded state and is
+ * within 2e-3 of the definition for the tokens that were chosen.
  */
 int cpmtp_sample_draft(const cpmtp_shape* shape, const void* h, const void* W_head, const void* E,
                        const void* W_g, const float* uniform, float temperature, int32_t topk,

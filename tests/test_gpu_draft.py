@@ -135,6 +135,21 @@ def test_long_runs_of_equal_scores_go_to_the_lowest_ids():
     assert np.max(np.abs(np.sort(out["topk_logp"].cpu().numpy(), axis=2) - np.sort(ref.topk_logp, axis=2))) <= LOGP_TOL
 
 
+def test_vocabulary_of_more_chunks_than_threads():
+    """V > 2048 * 256: the merging block's threads each hold the candidate lists of several chunks."""
+    from paper_2410_17765_b200 import binding
+
+    shape = synth.Shape(N=2, d=64, V=2048 * 256 + 5000, n=2, r=2)
+    inp = synth.make_inputs(shape, seed=13, weight_scale=8.0)
+    ref = cp_head.draft(inp.h, inp.W_head, inp.E, inp.W_g, shape.n, shape.r, topk=4)
+    st = torch.zeros(1, dtype=torch.int32, device="cuda")
+    out = binding.sample_draft(*to_dev(inp), shape.n, topk=4, dev_status=st)
+    torch.cuda.synchronize()
+    assert int(st.item()) == 0
+    frac = check_against_oracle(inp, out, ref, 4)
+    assert frac >= 0.75
+
+
 def test_verify_draft_matches_oracle():
     from paper_2410_17765_b200 import binding
 
