@@ -34,6 +34,7 @@ constexpr int kWideStages = 3;                        // 64 KB per slot
 constexpr int kWideBM = 2 * kBM;
 using CfgKKSkinny = TileCfg<kBN, 5, false, false, 32>;   // <= 32 rows of A: bandwidth-bound draft scoring
 using WideKK = TileCfg<kBN, kWideStages, false, false, kBM, 2>;   // 256 x 256 tiles, two row blocks share B
+using CfgProj = TileCfg<kBN, kStages, false, false, kBM, 1, 2>;   // 128-row tiles, eight epilogue warps (head projection)
 
 inline size_t align_up(size_t v, size_t a = kAlign) { return (v + a - 1) / a * a; }
 
@@ -595,9 +596,17 @@ int run_forward(const cpmtp_shape& s, const uint16_t* h, const uint16_t* W_head,
       const int n_tiles = (ncols + kBN - 1) / kBN;
       const Sched sc = make_sched(1, n_tiles, n_tiles, 1, s.d / kBK);
       CPMTP_TRY((launch_gemm<CfgKKSkinny, EpiProj<kBN>>(h, s.N, s.d, W_head, ncols, s.d, s.d, sc, ep, dev_status, sms, stream)));
-    } else {
+    } else if (knobs().proj_tiles == kBM || knobs().proj_tiles == kWideBM) {   // tuning knob: the plain tile shapes
       CPMTP_TRY((gemm_auto<false, false, EpiProj<kBN>>(h, s.d, W_head, s.d, s.N, ncols, s.d, 8192, ep, dev_status, sms, stream,
-                                                      static_cast<int>(knobs().proj_tiles))));   // knob: tuning only
+                                                      static_cast<int>(knobs().proj_tiles))));
+    } else {
+      // Its epilogue (bf16 slab stores, gathered rows of E, one partial per 64 columns) is a long dependent chain
+      // per chunk: with one warp per scheduler it, not the MMAs, sets the pace of a tile.  Two warps per TMEM lane
+      // quarter, each with half of the columns, on 128-row tiles whose accumulator is double-buffered.
+      const int n_tiles = (ncols + kBN - 1) / kBN;
+      const int m_tiles = (s.N + kBM - 1) / kBM;
+      const Sched sc = make_sched(m_tiles, n_tiles, n_tiles, 8192 / kBM, s.d / kBK);
+      CPMTP_TRY((launch_gemm<CfgProj, EpiProj<kBN>>(h, s.N, s.d, W_head, ncols, s.d, s.d, sc, ep, dev_status, sms, stream)));
     }
   }
   // unembedding fused with the vocabulary log-sum-exp (Eq. 6, Eq. 8)

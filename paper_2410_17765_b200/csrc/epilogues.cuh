@@ -188,12 +188,18 @@ struct EpiProj : EpiDefaults {
 
   __device__ static void tile(const Params& p, State& st, uint32_t tacc, int m_tile, int n_tile, int row_in_tile,
                               uint8_t* smem, int epi_tid) {
+    tile_part(p, st, tacc, m_tile, n_tile, row_in_tile, smem, epi_tid, 0, BN);
+  }
+  // Columns [c_begin, c_end) of the tile (multiples of 64): the whole tile, or the part of it that one of two
+  // warps on the same accumulator rows handles.
+  __device__ static void tile_part(const Params& p, State& st, uint32_t tacc, int m_tile, int n_tile, int row_in_tile,
+                                   uint8_t* smem, int epi_tid, int c_begin, int c_end) {
     const int row = m_tile * kBM + row_in_tile;
     const bool valid = row < p.M;
     const bool gather = valid && p.x != nullptr;
     const int tile_col0 = n_tile * BN;
-    const int c_hi = chunk_end(tile_col0, BN, p.ncols);
-    if (c_hi <= 0) return;
+    const int c_hi = chunk_end(tile_col0, c_end, p.ncols);
+    if (c_hi <= c_begin) return;
     // slice of the target row of E that chunk c multiplies: 32 bf16 = four 16-byte loads
     auto fetch = [&](int c, uint4 (&e)[4]) {
       if (!gather) return;
@@ -235,10 +241,10 @@ struct EpiProj : EpiDefaults {
     };
     float va[32], vb[32];
     uint4 ea[4], eb[4];
-    ptx::tmem_ld_32x32(tacc, va);
-    fetch(0, ea);
+    ptx::tmem_ld_32x32(tacc + c_begin, va);
+    fetch(c_begin, ea);
 #pragma unroll 1
-    for (int c = 0; c < c_hi; c += 64) {
+    for (int c = c_begin; c < c_hi; c += 64) {
       ptx::tmem_ld_wait_for(va);
       const bool more = c + 32 < c_hi;   // always true here (ncols % 64 == 0); kept for symmetry
       if (more) {

@@ -2,11 +2,14 @@
 //
 //   D[M, N] = A[M, K] * B[N, K]^T      bf16 operands, fp32 accumulation in TMEM
 //
-// One CTA per SM, 64 + 128*MB threads:
+// One CTA per SM, 64 + 128 * MB * EW threads:
 //   warp 0      TMA producer (one lane): global -> 128B-swizzled shared tiles
 //   warp 1      MMA issuer (one lane): tcgen05.mma, accumulators in TMEM
-//   then 4 epilogue warps per 128-row block: tcgen05.ld the 128 x BN fp32 block and
-//   hand it to `Epi` (a warp may read only the TMEM lane quarter given by warp id % 4)
+//   then 4 * EW epilogue warps per 128-row block: tcgen05.ld the 128 x BN fp32 block and
+//   hand it to `Epi` (a warp may read only the TMEM lane quarter given by warp id % 4).
+//   EW = 2 puts two warps on every lane quarter, each with half of the tile's columns: for
+//   epilogues whose per-chunk work is a long dependent chain (a single warp per scheduler
+//   cannot hide its own latencies) and that keep no state across chunks.
 // MB = 1: a 128 x BN tile, accumulator double-buffered in TMEM (2 x BN columns) so the
 //   epilogue of tile j overlaps the MMAs of tile j+1; ring slots of (128 x 64) A + (BN x 64) B.
 // MB = 2 ("wide"): a 256 x 256 tile as two 128-row blocks that share every B slot (two MMAs
@@ -125,19 +128,21 @@ __device__ __forceinline__ bool decode_unit(const Sched& s, int u, int& m_tile, 
 // that many rows of the A tile are fetched and given shared memory; the MMA still spans 128
 // rows and the accumulator rows beyond A_ROWS hold garbage that no epilogue may use.  The
 // space saved buys deeper pipelining of the B stream (bandwidth-bound draft scoring).
-template <int BN_, int STAGES_, bool A_MN_, bool B_MN_, int A_ROWS_ = kBM, int MB_ = 1>
+template <int BN_, int STAGES_, bool A_MN_, bool B_MN_, int A_ROWS_ = kBM, int MB_ = 1, int EW_ = 1>
 struct TileCfg {
   static constexpr int BN = BN_;
   static constexpr int STAGES = STAGES_;
   static constexpr bool A_MN = A_MN_;
   static constexpr bool B_MN = B_MN_;
   static constexpr int MB = MB_;                       // 128-row blocks per tile
+  static constexpr int EW = EW_;                       // epilogue warps per TMEM lane quarter of a row block
   static constexpr int A_ROWS = A_ROWS_;               // rows of A fetched per 128-row block
   static constexpr int TILE_M = kBM * MB;
   static constexpr int A_BLOCK_BYTES = A_ROWS * kBK * 2;
   static constexpr int A_BYTES = A_BLOCK_BYTES * MB;
   static constexpr int ACC_STAGES = MB == 1 ? 2 : 1;
-  static constexpr int THREADS = 64 + kEpiThreads * MB;
+  static constexpr int THREADS = 64 + kEpiThreads * MB * EW;
+  static_assert(EW == 1 || (EW == 2 && BN_ % 128 == 0), "column halves are whole 64-column blocks");
   static_assert(MB == 1 || MB == 2, "one or two 128-row blocks");
   static_assert(MB == 1 || (A_ROWS == kBM && BN == 256), "wide tiles are 256 x 256");
   static_assert(A_ROWS == kBM || (!A_MN_ && A_ROWS % 8 == 0 && A_ROWS >= 8), "skinny A needs a K-major A");
@@ -156,16 +161,16 @@ constexpr int kBarrierBytes = 256;
 
 template <class Cfg, class Epi>
 constexpr int gemm_smem_bytes() {
-  return 1024 + Cfg::STAGES * Cfg::STAGE_BYTES + kBarrierBytes + Epi::SMEM_PER_WARP * 4 * Cfg::MB;
+  return 1024 + Cfg::STAGES * Cfg::STAGE_BYTES + kBarrierBytes + Epi::SMEM_PER_WARP * 4 * Cfg::MB * Cfg::EW;
 }
 
 // Shared memory: [<= 1023 B alignment pad][STAGES operand slots][epilogue staging: Epi::SMEM_PER_WARP bytes for each
-// of the 4 * MB epilogue warps][barriers].
+// of the 4 * MB * EW epilogue warps][barriers].
 template <class Cfg, class Epi>
 __global__ void __launch_bounds__(Cfg::THREADS, 1)
 tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
                const Sched sched, const __grid_constant__ typename Epi::Params ep, int* __restrict__ dev_status) {
-  constexpr int kEpiSmem = Epi::SMEM_PER_WARP * 4 * Cfg::MB;
+  constexpr int kEpiSmem = Epi::SMEM_PER_WARP * 4 * Cfg::MB * Cfg::EW;
   static_assert(kEpiSmem % 1024 == 0, "epilogue staging keeps the 1024-byte alignment of the slots");
   static_assert(1024 + Cfg::STAGES * Cfg::STAGE_BYTES + kBarrierBytes + kEpiSmem <= 232448,
                 "more shared memory than a CTA can have");
@@ -198,7 +203,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     }
     for (int a = 0; a < 2; ++a) {
       ptx::mbar_init(tfull_bar(a), 1);
-      ptx::mbar_init(tempty_bar(a), kEpiThreads * Cfg::MB);
+      ptx::mbar_init(tempty_bar(a), kEpiThreads * Cfg::MB * Cfg::EW);
     }
     ptx::mbar_init(drain_bar, 1);
     *abort_flag = 0;
@@ -323,10 +328,12 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     // same barrier, so they either all pass or all time out, and no warp is left
     // alone at a barrier an epilogue might use internally.
     const int quarter = warp & 3;                 // TMEM lane quarter this warp may read
-    const int mblock = (warp - 2) >> 2;           // which 128-row block of the tile
+    const int wgroup = (warp - 2) >> 2;           // group of four warps: one row block, one column part
+    const int mblock = wgroup % Cfg::MB;          // which 128-row block of the tile
+    const int cpart = wgroup / Cfg::MB;           // which part of the tile's columns (EW > 1)
     const int row_in_tile = quarter * 32 + lane;  // row within that block
     const int epi_tid = (threadIdx.x - 64) & (kEpiThreads - 1);
-    uint8_t* my_smem = epi_smem + mblock * (Epi::SMEM_PER_WARP * 4);   // this row block's staging
+    uint8_t* my_smem = epi_smem + wgroup * (Epi::SMEM_PER_WARP * 4);   // this warp group's staging
     typename Epi::State st;
     int acc_it = 0;
     bool alive = true;
@@ -343,7 +350,12 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         ptx::tc_fence_after_sync();
         const uint32_t tacc = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16) +
                               (acc * Cfg::MB + mblock) * Cfg::BN;
-        Epi::tile(ep, st, tacc, m_block_tile, nt, row_in_tile, my_smem, epi_tid);
+        if constexpr (Cfg::EW == 1) {
+          Epi::tile(ep, st, tacc, m_block_tile, nt, row_in_tile, my_smem, epi_tid);
+        } else {
+          constexpr int kPart = Cfg::BN / Cfg::EW;
+          Epi::tile_part(ep, st, tacc, m_block_tile, nt, row_in_tile, my_smem, epi_tid, cpart * kPart, (cpart + 1) * kPart);
+        }
         ptx::tc_fence_before_sync();
         ptx::mbar_arrive(tempty_bar(acc));
       }
