@@ -47,6 +47,8 @@
  *    CPMTP_GEMM_GROUP_ROWS (rows swept together by the other GEMMs), CPMTP_WIDE_MIN_K
  *    and CPMTP_WIDE_MIN_ROWS (shortest contraction / fewest rows that get 256-row tiles), CPMTP_KL_GROUP_TILES and CPMTP_KL_SPLITS
  *    (schedule of the KL sweep of cpmtp_distill_forward; the latter also sizes its workspace),
+ *    CPMTP_PROJ_TILE_ROWS (128 or 256: run the head projection on the plain 128- or 256-row tiles with four
+ *    epilogue warps per row block instead of its own configuration),
  *    CPMTP_WAIT_LIMIT_US (how long a wait inside a kernel may last before the kernel gives up with
  *    device status 2; default 4 s) and CPMTP_TEST_SKIP_LOAD (test hook: every CTA of the tensor-core
  *    kernels leaves out that one operand load, so the give-up path runs; results are invalid).
