@@ -45,7 +45,8 @@ __device__ __forceinline__ bool cand_better(float s1, int i1, float s2, int i2) 
   return s1 > s2 || (s1 == s2 && i1 < i2);
 }
 
-// List of at most kMaxTopk candidates kept in registers; insert() keeps a list that is in order (best first) in order.
+// List of at most kMaxTopk candidates kept in registers.  insert() expects the list in order (best first) and
+// keeps it so; the other members accept any order.
 struct TopList {
   float score[kMaxTopk];
   int idx[kMaxTopk];

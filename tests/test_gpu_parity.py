@@ -188,6 +188,49 @@ def test_run_to_run_determinism():
         assert torch.equal(a, b)
 
 
+def test_calls_from_two_host_threads_on_their_own_streams():
+    """The header allows concurrent calls from several host threads when each has its own stream, workspace and
+    outputs (the host-side caches are behind a lock): two threads run forward + backward on different shapes at the
+    same time, repeatedly, and each gets bit for bit what it gets when it runs alone."""
+    import threading
+
+    from paper_2410_17765_b200 import binding
+
+    jobs = []
+    for name, seed in (("wide", 1), ("ragged", 2)):
+        shape = CASES[name]["shape"]
+        inp = synth.make_inputs(shape, seed=seed)
+        jobs.append((binding.make_shape(shape.N, shape.d, shape.V, shape.n, shape.r), to_dev(inp)))
+
+    def run(job, stream, reps, out):
+        cs, dev = job
+        with torch.cuda.stream(stream):
+            for _ in range(reps):
+                saved = binding.Saved.alloc(cs)
+                f = binding.forward(*dev, saved=saved)
+                g = binding.backward(*dev, saved)
+                stream.synchronize()
+                out.append((f["logp"].clone(), g["dh"].clone(), g["dW_head"].clone(), g["dE"].clone()))
+
+    alone = []
+    for job in jobs:
+        res = []
+        run(job, torch.cuda.Stream(), 1, res)
+        alone.append(res[0])
+    results = [[], []]
+    threads = [threading.Thread(target=run, args=(jobs[t], torch.cuda.Stream(), 6, results[t])) for t in range(2)]
+    for t in threads:
+        t.start()
+    for t in threads:
+        t.join()
+    torch.cuda.synchronize()
+    for t in range(2):
+        assert len(results[t]) == 6
+        for got in results[t]:
+            for a, b in zip(got, alone[t]):
+                assert torch.equal(a, b)
+
+
 def test_forward_host_matches_device_forward():
     from paper_2410_17765_b200 import binding
 
